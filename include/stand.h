@@ -1,0 +1,195 @@
+/* STAND speculative-sampling hot path for NVIDIA B200 (sm_100a): C interface.
+ *
+ * One decoding step passes once over the target logits of every draft-tree
+ * node (B sequences x N tree nodes x V vocabulary entries) and then
+ *   1. verifies the drafted tree by speculative sampling (paper Sec. 3.2 and
+ *      Sec. 4.2 "Stochastic tree drafting"),
+ *   2. feeds the accepted rows into the logit-based N-gram module (Sec. 4.1),
+ *   3. drafts the next tree from that module with Gumbel-Top-K (Sec. 4.2).
+ * The target model is not part of this library: logits are an input.
+ *
+ * Conventions
+ *   - Pointers named dev_* are DEVICE pointers, host_* are HOST pointers.  The
+ *     caller owns every buffer it passes, including the workspace; the library
+ *     keeps the workspace pointer until stand_destroy.
+ *   - `cu_stream` is a cudaStream_t passed as void* (NULL = default stream).
+ *     Calls that take a stream only enqueue work and return; they do not
+ *     synchronise unless stated.
+ *   - Return value: STAND_OK (0) or a negative STAND_E_* code.  Problems found
+ *     on the device (table full, probe limit, token id out of range) never trap:
+ *     they are counted and reported by stand_get_stats.
+ *   - Layouts are row-major, innermost dimension contiguous.
+ *   - Tree: node 0 is the root and carries the last token of the sequence;
+ *     parent[u] < u; nodes are numbered breadth-first so that the children of a
+ *     node are consecutive and ordered by draft rank.  Row (b,u) of the logits
+ *     is the target distribution of the token that FOLLOWS node u.
+ *   - Randomness: Philox4x32-10, key = seed, counter = (sequence, step, node,
+ *     slot), first output word, top 24 bits.  Slot j < 2^30: accept test of the
+ *     child of rank j; 0x40000000: the final sample of a walk; 0x80000000|t:
+ *     Gumbel noise of candidate token t.
+ */
+#ifndef STAND_H_
+#define STAND_H_
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+#define STAND_MAX_TOPK 12   /* entries kept per context (one 128-byte table slot) */
+#define STAND_MAX_ORDER 4   /* N-gram orders 1..4 (Sec. 4.1) */
+#define STAND_MAX_NODES 128 /* tree nodes per sequence */
+#define STAND_MAX_DEPTH 32
+#define STAND_MAX_VOCAB (1 << 20)
+
+#define STAND_DTYPE_F32 0
+#define STAND_DTYPE_BF16 1
+
+#define STAND_OK 0
+#define STAND_E_ARG (-1)       /* invalid argument or configuration */
+#define STAND_E_WORKSPACE (-2) /* workspace missing, misaligned or too small */
+#define STAND_E_CUDA (-3)      /* a CUDA runtime call failed */
+#define STAND_E_STATE (-4)     /* call not valid in the current state */
+
+typedef struct stand_ctx stand_ctx;
+
+typedef struct {
+  int32_t B;           /* sequences, >= 1 */
+  int32_t N;           /* tree nodes per sequence, root included, 1..STAND_MAX_NODES */
+  int32_t V;           /* vocabulary size, 2..STAND_MAX_VOCAB */
+  int32_t topk;        /* entries kept per context, 1..STAND_MAX_TOPK */
+  int32_t order_max;   /* N-gram orders 1..order_max, <= STAND_MAX_ORDER */
+  int32_t dtype;       /* STAND_DTYPE_* of the logits */
+  float temperature;   /* > 0 (Sec. 5: all sampling at temperature T) */
+  int32_t max_probe;   /* hash-table probe limit, >= 1 (0 = default 128) */
+  uint64_t seed;
+  uint64_t table_slots;   /* power of two, >= 2; one slot = 128 bytes */
+  const int32_t* parent;  /* HOST, [N]; parent[0] = -1; read during stand_init only */
+  int32_t chunks_per_unit; /* 0 = automatic; how many 1024-element chunks one warp streams */
+  int32_t host_staging;    /* != 0: reserve a logits staging buffer for stand_step_host */
+} stand_config;
+
+typedef struct {
+  uint64_t steps;           /* verifications run */
+  uint64_t emitted_tokens;  /* tokens emitted (accepted + sampled) */
+  uint64_t records;         /* (context, order) updates applied */
+  uint64_t inserts;         /* new contexts created */
+  uint64_t drops;           /* updates lost: probe limit reached / table full */
+  uint64_t bad_tokens;      /* token ids outside [0, V) met on the device */
+  uint64_t lookups;         /* drafting lookups (one per tree node with children) */
+  uint64_t lookup_hits[STAND_MAX_ORDER]; /* hits by order-1 */
+  uint64_t max_probe_seen;  /* longest probe sequence */
+} stand_stats;
+
+/* Bytes of device workspace a configuration needs; 0 if the configuration is invalid. */
+size_t stand_workspace_bytes(const stand_config* cfg);
+
+/* Creates a context in caller-owned device memory (256-byte aligned, at least
+ * stand_workspace_bytes).  Clears the N-gram tables, uploads the topology and
+ * synchronises the device once.  The sequences start empty: call
+ * stand_reset_sequences before the first step. */
+int stand_init(const stand_config* cfg, void* dev_workspace, size_t bytes, stand_ctx** out);
+
+/* Frees the host-side context.  Device memory stays with the caller. */
+int stand_destroy(stand_ctx* ctx);
+
+/* (Re)starts all sequences.  dev_tail [B, order_max] int32: the last tokens of each
+ * prompt, -1 padded at the front; dev_len [B] int64: tokens so far.  The N-gram
+ * tables are kept: the module persists across trajectories (Sec. 5.1).  The draft
+ * tree is cleared, so the next verification samples one token from the root row. */
+int stand_reset_sequences(stand_ctx* ctx, const int32_t* dev_tail, const int64_t* dev_len, void* cu_stream);
+
+/* Sec. 3.2 + Sec. 4.2: one pass over dev_logits [B, N, V] (temperature softmax
+ * statistics and per-row top-k), then the verification walk of every sequence:
+ * drafted children are tested in draft order with the speculative-sampling ratio
+ * (recursive rejection, residual target, rejected token removed from the draft
+ * distribution); at the stop node one token is drawn by inverse CDF in token order.
+ * Writes dev_emitted [B, D+1] int32 (-1 padded; D = tree depth) and dev_n_emitted
+ * [B] int32, advances the sequences and the step counter, and records the
+ * accepted rows for stand_ngram_update. */
+int stand_verify_tree(stand_ctx* ctx, const void* dev_logits, int32_t* dev_emitted, int32_t* dev_n_emitted,
+                      void* cu_stream);
+
+/* Sec. 4.1: feeds the rows accepted by the last verification into the tables,
+ * under every order 1..order_max whose context is available: a new context stores
+ * the row's top-k probabilities with count 1; a known one is averaged with weights
+ * c/(c+1) and 1/(c+1) (missing ids = 0), cut to the top-k, count c+1.  Updates are
+ * applied in (sequence, path position, order) order.  STAND_E_STATE if there is no
+ * pending verification. */
+int stand_ngram_update(stand_ctx* ctx, void* cu_stream);
+
+/* Sec. 4.1 without logits: M rows, each a context window (dev_ctx [M, order_max],
+ * the tokens before the predicted position, -1 padded at the front) and a
+ * compressed distribution (dev_ids [M, topk], -1 = unused; dev_probs [M, topk]);
+ * applied in row order, each under every order it is long enough for. */
+int stand_ngram_update_bulk(stand_ctx* ctx, const int32_t* dev_ctx, const int32_t* dev_ids, const float* dev_probs,
+                            int64_t M, void* cu_stream);
+
+/* Sec. 4.2: drafts the next tree of every sequence.  Breadth-first over the static
+ * topology; for a node with children the contexts of order order_max..1 are looked
+ * up, the first hit gives up to topk candidates (id, phi); the children are the
+ * candidates with the largest log(phi) - log(-log U) (Gumbel-Top-K), in that order.
+ * Nodes that cannot be drafted get -1.  Writes dev_tree_tokens [B, N] int32 (may be
+ * NULL) and keeps the tree and the candidate lists for the next verification. */
+int stand_draft_tree(stand_ctx* ctx, int32_t* dev_tree_tokens, void* cu_stream);
+
+/* verify -> update -> draft on one stream, no host synchronisation. */
+int stand_step(stand_ctx* ctx, const void* dev_logits, int32_t* dev_emitted, int32_t* dev_n_emitted,
+               int32_t* dev_tree_tokens, void* cu_stream);
+
+/* The same step for callers whose buffers live in HOST memory: copies host_logits
+ * [B, N, V] to the staging buffer (needs cfg.host_staging), runs the step, copies
+ * the three results back and synchronises the stream before returning. */
+int stand_step_host(stand_ctx* ctx, const void* host_logits, int32_t* host_emitted, int32_t* host_n_emitted,
+                    int32_t* host_tree_tokens, void* cu_stream);
+
+/* The row pass on its own (Sec. 5 temperature softmax, Sec. 4.1 top-k), without a
+ * context: for each of `rows` rows of dev_logits [rows, V] writes the log-sum-exp of
+ * x/T (dev_lse [rows] float), and the top-k entries by (value descending, id
+ * ascending): dev_ids [rows, topk] int32, dev_values [rows, topk] float (input
+ * values), dev_probs [rows, topk] float (softmax probabilities).  dev_scratch must
+ * hold stand_row_stats_scratch_bytes bytes, 256-byte aligned. */
+size_t stand_row_stats_scratch_bytes(int64_t rows, int32_t V, int32_t dtype, int32_t topk);
+int stand_row_stats(const void* dev_logits, int64_t rows, int32_t V, int32_t dtype, float temperature, int32_t topk,
+                    void* dev_scratch, size_t scratch_bytes, float* dev_lse, int32_t* dev_ids, float* dev_values,
+                    float* dev_probs, void* cu_stream);
+
+/* Synchronises the stream the context last used and copies the counters. */
+int stand_get_stats(stand_ctx* ctx, stand_stats* host_out);
+
+/* Results of the last verification, for inspection: accepted path dev_path [B, D+1]
+ * (node indices, -1 padded) and the compressed rows that will be fed to the tables,
+ * dev_ids / dev_probs [B, D+1, topk].  Any pointer may be NULL. */
+int stand_last_path(stand_ctx* ctx, int32_t* dev_path, int32_t* dev_ids, float* dev_probs, void* cu_stream);
+int32_t stand_tree_depth(const stand_ctx* ctx);
+
+/* Table export/import.  Device arrays: keys [cap, 4] int32 (-1 padded at the front),
+ * counts [cap] uint32, n_items [cap] int32, ids [cap, topk] int32, probs [cap, topk]
+ * float.  dump writes at most `cap` entries in arbitrary order and the total number
+ * of contexts to dev_total [1] uint64.  load inserts M entries (clear != 0 empties
+ * the tables first). */
+int stand_table_dump(stand_ctx* ctx, int32_t* dev_keys, uint32_t* dev_counts, int32_t* dev_n_items, int32_t* dev_ids,
+                     float* dev_probs, uint64_t cap, uint64_t* dev_total, void* cu_stream);
+int stand_table_load(stand_ctx* ctx, const int32_t* dev_keys, const uint32_t* dev_counts, const int32_t* dev_n_items,
+                     const int32_t* dev_ids, const float* dev_probs, uint64_t M, int32_t clear, void* cu_stream);
+
+/* Sequence state export/import (checkpoint/resume): tails [B, order_max], lengths
+ * [B] int64, tree tokens [B, N], candidate lists cand_n [B, N], cand_id / cand_phi
+ * [B, N, topk], and the step counter (host).  load discards a pending verification. */
+int stand_state_dump(stand_ctx* ctx, int32_t* dev_tail, int64_t* dev_len, int32_t* dev_tree, int32_t* dev_cand_n,
+                     int32_t* dev_cand_id, float* dev_cand_phi, uint32_t* host_step, void* cu_stream);
+int stand_state_load(stand_ctx* ctx, const int32_t* dev_tail, const int64_t* dev_len, const int32_t* dev_tree,
+                     const int32_t* dev_cand_n, const int32_t* dev_cand_id, const float* dev_cand_phi,
+                     uint32_t step, void* cu_stream);
+
+/* How many kernels the library has launched through this context so far. */
+uint64_t stand_launch_count(const stand_ctx* ctx);
+
+const char* stand_strerror(int code);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* STAND_H_ */

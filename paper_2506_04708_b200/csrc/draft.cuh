@@ -1,0 +1,121 @@
+// Stochastic tree drafting (paper Sec. 4.2).  One thread block per sequence walks
+// the static topology level by level; one warp per parent node:
+//   - the contexts of order n_max..1 of the would-be sequence (tail + path tokens)
+//     are probed at once, one lane per order; the longest hit wins ("first
+//     successful match", longest first);
+//   - the hit's candidates (id, phi) sit one per lane; Gumbel-Top-K: each lane
+//     forms g = log(phi) - log(-log U) with its own Philox uniform (keyed by the
+//     token id) and its rank among the candidates; rank r < #children becomes the
+//     child of draft rank r;
+//   - the candidate list is kept as the draft distribution for the next verification.
+#pragma once
+#include "common.cuh"
+#include "table.cuh"
+
+namespace stand {
+
+constexpr int K4_THREADS = 256;
+
+struct DraftParams {
+  const Slot* table;
+  unsigned long long mask;
+  int max_probe, B, N, K, n_max, D, V;
+  unsigned long long seed;
+  uint32_t step;
+  const int* parent;       // [N]
+  const int* first_child;  // [N]
+  const int* n_children;   // [N]
+  const int* level_start;  // [D+2]
+  const int* tail;         // [B, n_max]
+  int* tree;               // [B, N]
+  int* tree_user;          // [B, N] or null
+  int* cand_n;             // [B, N]
+  int* cand_id;            // [B, N, K]
+  float* cand_phi;         // [B, N, K]
+  unsigned long long* stats;
+};
+
+__global__ void __launch_bounds__(K4_THREADS) draft_kernel(const DraftParams p) {
+  __shared__ int s_tok[NODES_MAX];
+  const int b = blockIdx.x, tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+  const int N = p.N, K = p.K, n_max = p.n_max;
+  for (int u = tid; u < N; u += K4_THREADS) s_tok[u] = -1;
+  __syncthreads();
+  if (tid == 0) s_tok[0] = p.tail[b * n_max + n_max - 1];  // the root carries the last token
+  __syncthreads();
+
+  for (int d = 0; d < p.D; ++d) {
+    const int l0 = p.level_start[d], l1 = p.level_start[d + 1];
+    for (int u = l0 + warp; u < l1; u += K4_THREADS / 32) {
+      const int m = p.n_children[u];
+      const long long row = (long long)b * N + u;
+      if (m == 0) { if (lane == 0) p.cand_n[row] = 0; continue; }
+      const bool drafted = u == 0 || s_tok[u] >= 0;
+      if (!drafted) { if (lane == 0) p.cand_n[row] = 0; continue; }  // nothing is drafted below an undrafted node
+      // last n_max tokens of the sequence as it reads if the path root..u is accepted
+      int win[ORDER_MAX];
+      {
+        int filled = 0, w = u;
+        while (w != 0 && filled < n_max) { win[n_max - 1 - filled] = s_tok[w]; ++filled; w = p.parent[w]; }
+        for (int i = n_max - 1; filled < n_max; --i, ++filled) win[n_max - 1 - filled] = p.tail[b * n_max + i];
+      }
+      // one lane per order
+      uint32_t slot = NO_SLOT;
+      if (lane < n_max) {
+        const int n = lane + 1;
+        int key[4] = {-1, -1, -1, -1};
+        bool ok = true;
+        for (int i = 0; i < n; ++i) {
+          const int t = win[n_max - n + i];
+          if (t < 0 || t >= p.V) ok = false;
+          key[4 - n + i] = t;
+        }
+        if (ok) slot = find_slot(p.table, p.mask, p.max_probe, key);
+      }
+      const unsigned hits = __ballot_sync(FULL, slot != NO_SLOT);
+      if (lane == 0) {
+        atomicAdd(&p.stats[ST_LOOKUPS], 1ull);
+        if (hits) atomicAdd(&p.stats[ST_HIT0 + (31 - __clz(hits))], 1ull);
+      }
+      if (hits == 0) { if (lane == 0) p.cand_n[row] = 0; continue; }
+      const int winner = 31 - __clz(hits);  // the longest order that matched
+      slot = __shfl_sync(FULL, slot, winner);
+      const Slot* s = &p.table[slot];
+      const int n_items = (int)s->n_items;
+      int id = -1;
+      float phi = 0.0f;
+      if (lane < n_items && lane < K) { id = s->ids[lane]; phi = s->probs[lane]; }
+      const bool valid = id >= 0 && phi > 0.0f;
+      double g = 0.0;
+      if (valid) {
+        const double U = ((double)philox_u24(p.seed, b, p.step, u, SLOT_GUMBEL | (uint32_t)id) + 0.5) * (1.0 / 16777216.0);
+        g = log((double)phi) - log(-log(U));
+      }
+      int rank = 0;
+      for (int j = 0; j < KMAX; ++j) {
+        const double gj = __shfl_sync(FULL, g, j);
+        const int idj = __shfl_sync(FULL, id, j);
+        const bool vj = __shfl_sync(FULL, (int)valid, j) != 0;
+        if (vj && (gj > g || (gj == g && idj < id))) ++rank;
+      }
+      if (valid && rank < m) s_tok[p.first_child[u] + rank] = id;
+      const unsigned vmask = __ballot_sync(FULL, valid);
+      if (valid) {
+        const int pos = __popc(vmask & ((1u << lane) - 1u));
+        p.cand_id[row * K + pos] = id;
+        p.cand_phi[row * K + pos] = phi;
+      }
+      if (lane == 0) p.cand_n[row] = __popc(vmask);
+    }
+    __syncthreads();
+  }
+  // nodes of the deepest level have no children
+  for (int u = p.level_start[p.D] + tid; u < N; u += K4_THREADS) p.cand_n[(long long)b * N + u] = 0;
+  for (int u = tid; u < N; u += K4_THREADS) {
+    const int t = s_tok[u];
+    p.tree[(long long)b * N + u] = t;
+    if (p.tree_user) p.tree_user[(long long)b * N + u] = t;
+  }
+}
+
+}  // namespace stand

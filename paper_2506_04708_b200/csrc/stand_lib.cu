@@ -1,0 +1,554 @@
+// C interface of the STAND CUDA library: context, workspace layout, launches.
+// Declarations and the meaning of every argument: include/stand.h.
+#include "../../include/stand.h"
+
+#include <cuda_runtime.h>
+#include <new>
+#include <stdio.h>
+#include <string.h>
+
+#include "common.cuh"
+#include "draft.cuh"
+#include "row_pass.cuh"
+#include "table.cuh"
+#include "verify.cuh"
+
+using namespace stand;
+
+namespace {
+
+constexpr int BULK_ROWS = 2048;  // rows per batch of the bulk update
+
+struct Layout {
+  size_t table, topo, tail, len, tree, cand_n, cand_id, cand_phi, pairs, part, emitted, n_path, path, rec_ctx, rec_ids,
+      rec_p, rec_slot, stats, scratch64, staging, total;
+};
+
+inline size_t align_up(size_t x) { return (x + 255) & ~(size_t)255; }
+
+struct Derived {
+  int D, n_chunks, cpu, upr;
+  int parent[NODES_MAX], first_child[NODES_MAX], n_children[NODES_MAX], depth[NODES_MAX], level_start[DEPTH_MAX + 2];
+};
+
+bool derive(const stand_config* c, Derived* d) {
+  if (!c) return false;
+  if (c->B < 1 || c->N < 1 || c->N > STAND_MAX_NODES || c->V < 2 || c->V > STAND_MAX_VOCAB) return false;
+  if (c->topk < 1 || c->topk > STAND_MAX_TOPK || c->order_max < 1 || c->order_max > STAND_MAX_ORDER) return false;
+  if (c->dtype != STAND_DTYPE_F32 && c->dtype != STAND_DTYPE_BF16) return false;
+  if (!(c->temperature > 0.0f) || c->max_probe < 0 || c->chunks_per_unit < 0) return false;
+  if (c->table_slots < 2 || (c->table_slots & (c->table_slots - 1)) != 0 || c->table_slots > (1ull << 32) - 2) return false;
+  if (!c->parent || c->parent[0] != -1) return false;
+  if ((long long)c->B * c->N > (1ll << 31) / 4) return false;
+  memset(d, 0, sizeof(*d));
+  d->parent[0] = -1;
+  d->D = 0;
+  for (int u = 0; u < c->N; ++u) d->first_child[u] = -1;
+  for (int u = 1; u < c->N; ++u) {
+    const int par = c->parent[u];
+    if (par < 0 || par >= u) return false;
+    if (u > 1 && par < c->parent[u - 1]) return false;  // breadth-first numbering, siblings contiguous
+    d->parent[u] = par;
+    d->depth[u] = d->depth[par] + 1;
+    if (d->depth[u] < d->depth[u - 1]) return false;
+    if (d->depth[u] > STAND_MAX_DEPTH) return false;
+    if (d->first_child[par] < 0) d->first_child[par] = u;
+    d->n_children[par] += 1;
+    if (d->depth[u] > d->D) d->D = d->depth[u];
+  }
+  for (int u = 0; u < c->N; ++u)
+    if (d->first_child[u] < 0) d->first_child[u] = 0;
+  for (int l = 0; l <= d->D + 1; ++l) d->level_start[l] = c->N;
+  for (int u = c->N - 1; u >= 0; --u) d->level_start[d->depth[u]] = u;
+  d->n_chunks = (c->V + CHUNK - 1) / CHUNK;
+  if (c->chunks_per_unit > 0) d->cpu = c->chunks_per_unit < d->n_chunks ? c->chunks_per_unit : d->n_chunks;
+  else {
+    // enough units to fill 148 SMs x 24 warps about twice over, units as long as that allows
+    const long long total = (long long)c->B * c->N * d->n_chunks;
+    long long cpu = (total + 7103) / 7104;
+    if (cpu < 1) cpu = 1;
+    if (cpu > d->n_chunks) cpu = d->n_chunks;
+    d->cpu = (int)cpu;
+  }
+  d->upr = (d->n_chunks + d->cpu - 1) / d->cpu;
+  return true;
+}
+
+size_t esize_of(int dtype) { return dtype == STAND_DTYPE_F32 ? 4 : 2; }
+
+void layout_of(const stand_config* c, const Derived* d, Layout* L) {
+  const size_t B = c->B, N = c->N, K = c->topk, W = d->D + 1, n = c->order_max;
+  size_t rec_rows = B * W;
+  if (rec_rows < (size_t)BULK_ROWS) rec_rows = BULK_ROWS;
+  size_t at = 0;
+  auto take = [&](size_t bytes) { const size_t here = at; at = align_up(at + bytes); return here; };
+  L->table = take((size_t)c->table_slots * sizeof(Slot));
+  L->topo = take((4 * NODES_MAX + DEPTH_MAX + 2) * sizeof(int));
+  L->tail = take(B * n * 4);
+  L->len = take(B * 8);
+  L->tree = take(B * N * 4);
+  L->cand_n = take(B * N * 4);
+  L->cand_id = take(B * N * K * 4);
+  L->cand_phi = take(B * N * K * 4);
+  L->pairs = take(B * N * (size_t)d->n_chunks * sizeof(float2));
+  L->part = take(B * N * (size_t)d->upr * K * sizeof(uint2));
+  L->emitted = take(B * W * 4);
+  L->n_path = take(B * 4);
+  L->path = take(B * W * 4);
+  L->rec_ctx = take(B * W * n * 4);
+  L->rec_ids = take(B * W * K * 4);
+  L->rec_p = take(B * W * K * 4);
+  L->rec_slot = take(rec_rows * n * 4);
+  L->stats = take(ST_COUNT * 8);
+  L->scratch64 = take(64);
+  L->staging = take(c->host_staging ? B * N * (size_t)c->V * esize_of(c->dtype) : 0);
+  L->total = at;
+}
+
+}  // namespace
+
+struct stand_ctx {
+  stand_config cfg;
+  Derived d;
+  Layout L;
+  char* ws;
+  uint32_t step;
+  bool pending;
+  uint64_t launches;
+  cudaStream_t last_stream;
+  int max_probe;
+  float c;  // log2(e) / T
+
+  template <typename T> T* at(size_t off) const { return reinterpret_cast<T*>(ws + off); }
+  int* topo_parent() const { return at<int>(L.topo); }
+  int* topo_first_child() const { return at<int>(L.topo) + NODES_MAX; }
+  int* topo_n_children() const { return at<int>(L.topo) + 2 * NODES_MAX; }
+  int* topo_depth() const { return at<int>(L.topo) + 3 * NODES_MAX; }
+  int* topo_level_start() const { return at<int>(L.topo) + 4 * NODES_MAX; }
+};
+
+namespace {
+
+int cuda_ok(cudaError_t e) { return e == cudaSuccess ? STAND_OK : STAND_E_CUDA; }
+int launch_ok() { return cuda_ok(cudaGetLastError()); }
+
+float log2e_over_T(float T) { return (float)(1.4426950408889634 / (double)T); }
+
+bool rows_aligned(const void* base, int V, int dtype) {
+  const size_t es = esize_of(dtype);
+  return ((uintptr_t)base % 16 == 0) && (((size_t)V * es) % 16 == 0);
+}
+
+int launch_row_pass(const void* logits, long long rows, int V, int dtype, int n_chunks, int cpu, int upr, float c, int topk,
+                    float2* pairs, uint2* part, cudaStream_t st) {
+  RowPassParams rp;
+  rp.logits = logits; rp.rows = rows; rp.V = V; rp.n_chunks = n_chunks; rp.cpu = cpu; rp.upr = upr; rp.c = c;
+  rp.topk = topk; rp.pairs = pairs; rp.part = part;
+  const long long units = rows * upr;
+  const long long blocks = (units + K1_WARPS - 1) / K1_WARPS;
+  if (blocks <= 0 || blocks > 0x7FFFFFFFll) return STAND_E_ARG;
+  const bool al = rows_aligned(logits, V, dtype);
+  if (dtype == STAND_DTYPE_BF16) {
+    if (al) row_pass_kernel<1, true><<<(unsigned)blocks, K1_THREADS, 0, st>>>(rp);
+    else row_pass_kernel<1, false><<<(unsigned)blocks, K1_THREADS, 0, st>>>(rp);
+  } else {
+    if (al) row_pass_kernel<0, true><<<(unsigned)blocks, K1_THREADS, 0, st>>>(rp);
+    else row_pass_kernel<0, false><<<(unsigned)blocks, K1_THREADS, 0, st>>>(rp);
+  }
+  return launch_ok();
+}
+
+int run_verify(stand_ctx* x, const void* logits, int32_t* emitted, int32_t* n_emitted, cudaStream_t st) {
+  const stand_config& c = x->cfg;
+  int rc = launch_row_pass(logits, (long long)c.B * c.N, c.V, c.dtype, x->d.n_chunks, x->d.cpu, x->d.upr, x->c, c.topk,
+                           x->at<float2>(x->L.pairs), x->at<uint2>(x->L.part), st);
+  if (rc) return rc;
+  x->launches += 1;
+  x->step += 1;  // the tree drafted in step s-1 is verified in step s
+  VerifyParams v;
+  v.logits = logits; v.dtype = c.dtype; v.B = c.B; v.N = c.N; v.V = c.V; v.K = c.topk; v.n_max = c.order_max;
+  v.D = x->d.D; v.n_chunks = x->d.n_chunks; v.upr = x->d.upr; v.c = x->c; v.seed = c.seed; v.step = x->step;
+  v.first_child = x->topo_first_child(); v.n_children = x->topo_n_children();
+  v.pairs = x->at<float2>(x->L.pairs); v.part = x->at<uint2>(x->L.part);
+  v.tail = x->at<int>(x->L.tail); v.len = x->at<long long>(x->L.len); v.tree = x->at<int>(x->L.tree);
+  v.cand_n = x->at<int>(x->L.cand_n); v.cand_id = x->at<int>(x->L.cand_id); v.cand_phi = x->at<float>(x->L.cand_phi);
+  v.emitted_user = emitted; v.n_emitted_user = n_emitted;
+  v.emitted = x->at<int>(x->L.emitted); v.n_path = x->at<int>(x->L.n_path); v.path = x->at<int>(x->L.path);
+  v.rec_ctx = x->at<int>(x->L.rec_ctx); v.rec_ids = x->at<int>(x->L.rec_ids); v.rec_p = x->at<float>(x->L.rec_p);
+  v.stats = x->at<unsigned long long>(x->L.stats);
+  verify_kernel<<<c.B, K2_THREADS, 0, st>>>(v);
+  rc = launch_ok();
+  if (rc) return rc;
+  x->launches += 1;
+  x->pending = true;
+  return STAND_OK;
+}
+
+int run_update_rows(stand_ctx* x, long long n_rows, const int* ctxw, const int* ids, const float* probs, const int* n_path,
+                    int width, cudaStream_t st) {
+  const stand_config& c = x->cfg;
+  UpdateParams u;
+  u.table = x->at<Slot>(x->L.table); u.mask = c.table_slots - 1; u.max_probe = x->max_probe; u.V = c.V; u.K = c.topk;
+  u.n_max = c.order_max; u.n_rows = n_rows; u.rec_ctx = ctxw; u.rec_ids = ids; u.rec_p = probs; u.n_path = n_path;
+  u.width = width; u.rec_slot = x->at<uint32_t>(x->L.rec_slot); u.stats = x->at<unsigned long long>(x->L.stats);
+  const long long n_rec = n_rows * c.order_max;
+  const unsigned blocks = (unsigned)((n_rec + 255) / 256);
+  update_locate_kernel<<<blocks, 256, 0, st>>>(u);
+  int rc = launch_ok();
+  if (rc) return rc;
+  update_apply_kernel<<<blocks, 256, 0, st>>>(u);
+  rc = launch_ok();
+  if (rc) return rc;
+  x->launches += 2;
+  return STAND_OK;
+}
+
+int run_update(stand_ctx* x, cudaStream_t st) {
+  const stand_config& c = x->cfg;
+  const int W = x->d.D + 1;
+  const int rc = run_update_rows(x, (long long)c.B * W, x->at<int>(x->L.rec_ctx), x->at<int>(x->L.rec_ids),
+                                 x->at<float>(x->L.rec_p), x->at<int>(x->L.n_path), W, st);
+  if (rc == STAND_OK) x->pending = false;
+  return rc;
+}
+
+int run_draft(stand_ctx* x, int32_t* tree_user, cudaStream_t st) {
+  const stand_config& c = x->cfg;
+  DraftParams d;
+  d.table = x->at<Slot>(x->L.table); d.mask = c.table_slots - 1; d.max_probe = x->max_probe; d.B = c.B; d.N = c.N;
+  d.K = c.topk; d.n_max = c.order_max; d.D = x->d.D; d.V = c.V; d.seed = c.seed; d.step = x->step;
+  d.parent = x->topo_parent(); d.first_child = x->topo_first_child(); d.n_children = x->topo_n_children();
+  d.level_start = x->topo_level_start(); d.tail = x->at<int>(x->L.tail); d.tree = x->at<int>(x->L.tree);
+  d.tree_user = tree_user; d.cand_n = x->at<int>(x->L.cand_n); d.cand_id = x->at<int>(x->L.cand_id);
+  d.cand_phi = x->at<float>(x->L.cand_phi); d.stats = x->at<unsigned long long>(x->L.stats);
+  draft_kernel<<<c.B, K4_THREADS, 0, st>>>(d);
+  const int rc = launch_ok();
+  if (rc == STAND_OK) x->launches += 1;
+  return rc;
+}
+
+__global__ void reset_tree_kernel(int B, int N, int n_max, const int* tail, int* tree, int* cand_n) {
+  const long long i = (long long)blockIdx.x * blockDim.x + threadIdx.x;
+  if (i >= (long long)B * N) return;
+  const int b = (int)(i / N), u = (int)(i % N);
+  tree[i] = u == 0 ? tail[b * n_max + n_max - 1] : -1;
+  cand_n[i] = 0;
+}
+
+}  // namespace
+
+extern "C" {
+
+size_t stand_workspace_bytes(const stand_config* cfg) {
+  Derived d;
+  if (!derive(cfg, &d)) return 0;
+  Layout L;
+  layout_of(cfg, &d, &L);
+  return L.total;
+}
+
+int stand_init(const stand_config* cfg, void* dev_workspace, size_t bytes, stand_ctx** out) {
+  if (!out) return STAND_E_ARG;
+  *out = nullptr;
+  Derived d;
+  if (!derive(cfg, &d)) return STAND_E_ARG;
+  Layout L;
+  layout_of(cfg, &d, &L);
+  if (!dev_workspace || ((uintptr_t)dev_workspace & 255) != 0 || bytes < L.total) return STAND_E_WORKSPACE;
+  stand_ctx* x = new (std::nothrow) stand_ctx;
+  if (!x) return STAND_E_ARG;
+  x->cfg = *cfg;
+  x->cfg.parent = nullptr;  // the host array is not kept
+  x->d = d;
+  x->L = L;
+  x->ws = (char*)dev_workspace;
+  x->step = 0;
+  x->pending = false;
+  x->launches = 0;
+  x->last_stream = 0;
+  x->max_probe = cfg->max_probe > 0 ? cfg->max_probe : 128;
+  x->c = log2e_over_T(cfg->temperature);
+
+  int topo[4 * NODES_MAX + DEPTH_MAX + 2];
+  memset(topo, 0, sizeof(topo));
+  memcpy(topo, d.parent, sizeof(d.parent));
+  memcpy(topo + NODES_MAX, d.first_child, sizeof(d.first_child));
+  memcpy(topo + 2 * NODES_MAX, d.n_children, sizeof(d.n_children));
+  memcpy(topo + 3 * NODES_MAX, d.depth, sizeof(d.depth));
+  memcpy(topo + 4 * NODES_MAX, d.level_start, sizeof(d.level_start));
+  int rc = cuda_ok(cudaMemcpy(x->ws + L.topo, topo, sizeof(topo), cudaMemcpyHostToDevice));
+  if (rc == STAND_OK) {
+    const unsigned long long n16 = (unsigned long long)cfg->table_slots * 8;
+    table_clear_kernel<<<(unsigned)((n16 + 255) / 256), 256>>>(x->at<Slot>(L.table), cfg->table_slots);
+    rc = launch_ok();
+  }
+  // everything after the table starts at zero, tails at -1
+  if (rc == STAND_OK) rc = cuda_ok(cudaMemset(x->ws + L.tail, 0xFF, L.len - L.tail));
+  if (rc == STAND_OK) rc = cuda_ok(cudaMemset(x->ws + L.len, 0, L.staging - L.len));
+  if (rc == STAND_OK) rc = cuda_ok(cudaMemset(x->ws + L.tree, 0xFF, L.cand_n - L.tree));
+  if (rc == STAND_OK) rc = cuda_ok(cudaDeviceSynchronize());
+  if (rc != STAND_OK) { delete x; return rc; }
+  x->launches += 1;
+  *out = x;
+  return STAND_OK;
+}
+
+int stand_destroy(stand_ctx* ctx) {
+  if (!ctx) return STAND_E_ARG;
+  delete ctx;
+  return STAND_OK;
+}
+
+int stand_reset_sequences(stand_ctx* x, const int32_t* dev_tail, const int64_t* dev_len, void* cu_stream) {
+  if (!x || !dev_tail || !dev_len) return STAND_E_ARG;
+  cudaStream_t st = (cudaStream_t)cu_stream;
+  x->last_stream = st;
+  const stand_config& c = x->cfg;
+  int rc = cuda_ok(cudaMemcpyAsync(x->ws + x->L.tail, dev_tail, (size_t)c.B * c.order_max * 4, cudaMemcpyDeviceToDevice, st));
+  if (rc) return rc;
+  rc = cuda_ok(cudaMemcpyAsync(x->ws + x->L.len, dev_len, (size_t)c.B * 8, cudaMemcpyDeviceToDevice, st));
+  if (rc) return rc;
+  const long long n = (long long)c.B * c.N;
+  reset_tree_kernel<<<(unsigned)((n + 255) / 256), 256, 0, st>>>(c.B, c.N, c.order_max, x->at<int>(x->L.tail),
+                                                                 x->at<int>(x->L.tree), x->at<int>(x->L.cand_n));
+  rc = launch_ok();
+  if (rc) return rc;
+  x->launches += 1;
+  x->pending = false;
+  return STAND_OK;
+}
+
+int stand_verify_tree(stand_ctx* x, const void* dev_logits, int32_t* dev_emitted, int32_t* dev_n_emitted, void* cu_stream) {
+  if (!x || !dev_logits) return STAND_E_ARG;
+  x->last_stream = (cudaStream_t)cu_stream;
+  return run_verify(x, dev_logits, dev_emitted, dev_n_emitted, (cudaStream_t)cu_stream);
+}
+
+int stand_ngram_update(stand_ctx* x, void* cu_stream) {
+  if (!x) return STAND_E_ARG;
+  if (!x->pending) return STAND_E_STATE;
+  x->last_stream = (cudaStream_t)cu_stream;
+  return run_update(x, (cudaStream_t)cu_stream);
+}
+
+int stand_ngram_update_bulk(stand_ctx* x, const int32_t* dev_ctx, const int32_t* dev_ids, const float* dev_probs, int64_t M,
+                            void* cu_stream) {
+  if (!x || M < 0 || (M > 0 && (!dev_ctx || !dev_ids || !dev_probs))) return STAND_E_ARG;
+  cudaStream_t st = (cudaStream_t)cu_stream;
+  x->last_stream = st;
+  const stand_config& c = x->cfg;
+  for (int64_t at = 0; at < M; at += BULK_ROWS) {
+    const long long n = M - at < BULK_ROWS ? M - at : BULK_ROWS;
+    const int rc = run_update_rows(x, n, dev_ctx + at * c.order_max, dev_ids + at * c.topk, dev_probs + at * c.topk,
+                                   nullptr, 1, st);
+    if (rc) return rc;
+  }
+  return STAND_OK;
+}
+
+int stand_draft_tree(stand_ctx* x, int32_t* dev_tree_tokens, void* cu_stream) {
+  if (!x) return STAND_E_ARG;
+  x->last_stream = (cudaStream_t)cu_stream;
+  return run_draft(x, dev_tree_tokens, (cudaStream_t)cu_stream);
+}
+
+int stand_step(stand_ctx* x, const void* dev_logits, int32_t* dev_emitted, int32_t* dev_n_emitted, int32_t* dev_tree_tokens,
+               void* cu_stream) {
+  if (!x || !dev_logits) return STAND_E_ARG;
+  cudaStream_t st = (cudaStream_t)cu_stream;
+  x->last_stream = st;
+  int rc = run_verify(x, dev_logits, dev_emitted, dev_n_emitted, st);
+  if (rc) return rc;
+  rc = run_update(x, st);
+  if (rc) return rc;
+  return run_draft(x, dev_tree_tokens, st);
+}
+
+int stand_step_host(stand_ctx* x, const void* host_logits, int32_t* host_emitted, int32_t* host_n_emitted,
+                    int32_t* host_tree_tokens, void* cu_stream) {
+  if (!x || !host_logits) return STAND_E_ARG;
+  if (!x->cfg.host_staging) return STAND_E_STATE;
+  cudaStream_t st = (cudaStream_t)cu_stream;
+  x->last_stream = st;
+  const stand_config& c = x->cfg;
+  const size_t bytes = (size_t)c.B * c.N * c.V * esize_of(c.dtype);
+  int rc = cuda_ok(cudaMemcpyAsync(x->ws + x->L.staging, host_logits, bytes, cudaMemcpyHostToDevice, st));
+  if (rc) return rc;
+  rc = run_verify(x, x->ws + x->L.staging, nullptr, nullptr, st);
+  if (rc) return rc;
+  rc = run_update(x, st);
+  if (rc) return rc;
+  rc = run_draft(x, nullptr, st);
+  if (rc) return rc;
+  const size_t W = x->d.D + 1;
+  if (host_emitted) rc = cuda_ok(cudaMemcpyAsync(host_emitted, x->ws + x->L.emitted, c.B * W * 4, cudaMemcpyDeviceToHost, st));
+  if (rc) return rc;
+  if (host_n_emitted) rc = cuda_ok(cudaMemcpyAsync(host_n_emitted, x->ws + x->L.n_path, (size_t)c.B * 4, cudaMemcpyDeviceToHost, st));
+  if (rc) return rc;
+  if (host_tree_tokens) rc = cuda_ok(cudaMemcpyAsync(host_tree_tokens, x->ws + x->L.tree, (size_t)c.B * c.N * 4, cudaMemcpyDeviceToHost, st));
+  if (rc) return rc;
+  return cuda_ok(cudaStreamSynchronize(st));
+}
+
+size_t stand_row_stats_scratch_bytes(int64_t rows, int32_t V, int32_t dtype, int32_t topk) {
+  if (rows < 1 || V < 2 || V > STAND_MAX_VOCAB || topk < 1 || topk > STAND_MAX_TOPK) return 0;
+  if (dtype != STAND_DTYPE_F32 && dtype != STAND_DTYPE_BF16) return 0;
+  const size_t n_chunks = (V + CHUNK - 1) / CHUNK;
+  // one unit per chunk at most
+  return align_up((size_t)rows * n_chunks * sizeof(float2)) + align_up((size_t)rows * n_chunks * topk * sizeof(uint2));
+}
+
+int stand_row_stats(const void* dev_logits, int64_t rows, int32_t V, int32_t dtype, float temperature, int32_t topk,
+                    void* dev_scratch, size_t scratch_bytes, float* dev_lse, int32_t* dev_ids, float* dev_values,
+                    float* dev_probs, void* cu_stream) {
+  const size_t need = stand_row_stats_scratch_bytes(rows, V, dtype, topk);
+  if (need == 0 || !dev_logits || !dev_lse || !dev_ids || !dev_values || !dev_probs || !(temperature > 0.0f)) return STAND_E_ARG;
+  if (!dev_scratch || ((uintptr_t)dev_scratch & 255) != 0 || scratch_bytes < need) return STAND_E_WORKSPACE;
+  cudaStream_t st = (cudaStream_t)cu_stream;
+  const int n_chunks = (V + CHUNK - 1) / CHUNK;
+  long long cpu = ((long long)rows * n_chunks + 7103) / 7104;
+  if (cpu < 1) cpu = 1;
+  if (cpu > n_chunks) cpu = n_chunks;
+  const int upr = (int)((n_chunks + cpu - 1) / cpu);
+  float2* pairs = (float2*)dev_scratch;
+  uint2* part = (uint2*)((char*)dev_scratch + align_up((size_t)rows * n_chunks * sizeof(float2)));
+  const float c = log2e_over_T(temperature);
+  int rc = launch_row_pass(dev_logits, rows, V, dtype, n_chunks, (int)cpu, upr, c, topk, pairs, part, st);
+  if (rc) return rc;
+  RowFinalizeParams f;
+  f.pairs = pairs; f.part = part; f.rows = rows; f.n_chunks = n_chunks; f.upr = upr; f.topk = topk; f.c = c;
+  f.lse = dev_lse; f.ids = dev_ids; f.values = dev_values; f.probs = dev_probs;
+  row_finalize_kernel<<<(unsigned)((rows + 7) / 8), 256, 0, st>>>(f);
+  return launch_ok();
+}
+
+int stand_get_stats(stand_ctx* x, stand_stats* host_out) {
+  if (!x || !host_out) return STAND_E_ARG;
+  int rc = cuda_ok(cudaStreamSynchronize(x->last_stream));
+  if (rc) return rc;
+  unsigned long long s[ST_COUNT];
+  rc = cuda_ok(cudaMemcpy(s, x->ws + x->L.stats, sizeof(s), cudaMemcpyDeviceToHost));
+  if (rc) return rc;
+  host_out->steps = s[ST_STEPS];
+  host_out->emitted_tokens = s[ST_EMITTED];
+  host_out->records = s[ST_RECORDS];
+  host_out->inserts = s[ST_INSERTS];
+  host_out->drops = s[ST_DROPS];
+  host_out->bad_tokens = s[ST_BAD_TOKENS];
+  host_out->lookups = s[ST_LOOKUPS];
+  for (int i = 0; i < STAND_MAX_ORDER; ++i) host_out->lookup_hits[i] = s[ST_HIT0 + i];
+  host_out->max_probe_seen = s[ST_MAX_PROBE];
+  return STAND_OK;
+}
+
+int stand_last_path(stand_ctx* x, int32_t* dev_path, int32_t* dev_ids, float* dev_probs, void* cu_stream) {
+  if (!x) return STAND_E_ARG;
+  cudaStream_t st = (cudaStream_t)cu_stream;
+  x->last_stream = st;
+  const stand_config& c = x->cfg;
+  const size_t W = x->d.D + 1;
+  int rc = STAND_OK;
+  if (dev_path) rc = cuda_ok(cudaMemcpyAsync(dev_path, x->ws + x->L.path, c.B * W * 4, cudaMemcpyDeviceToDevice, st));
+  if (rc == STAND_OK && dev_ids) rc = cuda_ok(cudaMemcpyAsync(dev_ids, x->ws + x->L.rec_ids, c.B * W * c.topk * 4, cudaMemcpyDeviceToDevice, st));
+  if (rc == STAND_OK && dev_probs) rc = cuda_ok(cudaMemcpyAsync(dev_probs, x->ws + x->L.rec_p, c.B * W * c.topk * 4, cudaMemcpyDeviceToDevice, st));
+  return rc;
+}
+
+int32_t stand_tree_depth(const stand_ctx* x) { return x ? x->d.D : -1; }
+
+int stand_table_dump(stand_ctx* x, int32_t* dev_keys, uint32_t* dev_counts, int32_t* dev_n_items, int32_t* dev_ids,
+                     float* dev_probs, uint64_t cap, uint64_t* dev_total, void* cu_stream) {
+  if (!x || !dev_total || (cap > 0 && (!dev_keys || !dev_counts || !dev_n_items || !dev_ids || !dev_probs))) return STAND_E_ARG;
+  cudaStream_t st = (cudaStream_t)cu_stream;
+  x->last_stream = st;
+  int rc = cuda_ok(cudaMemsetAsync(dev_total, 0, 8, st));
+  if (rc) return rc;
+  const unsigned long long n = x->cfg.table_slots;
+  table_dump_kernel<<<(unsigned)((n + 255) / 256), 256, 0, st>>>(x->at<Slot>(x->L.table), n, x->cfg.topk, dev_keys, dev_counts,
+                                                                 dev_n_items, dev_ids, dev_probs, cap,
+                                                                 (unsigned long long*)dev_total);
+  rc = launch_ok();
+  if (rc == STAND_OK) x->launches += 1;
+  return rc;
+}
+
+int stand_table_load(stand_ctx* x, const int32_t* dev_keys, const uint32_t* dev_counts, const int32_t* dev_n_items,
+                     const int32_t* dev_ids, const float* dev_probs, uint64_t M, int32_t clear, void* cu_stream) {
+  if (!x || (M > 0 && (!dev_keys || !dev_counts || !dev_n_items || !dev_ids || !dev_probs))) return STAND_E_ARG;
+  cudaStream_t st = (cudaStream_t)cu_stream;
+  x->last_stream = st;
+  int rc = STAND_OK;
+  if (clear) {
+    const unsigned long long n16 = (unsigned long long)x->cfg.table_slots * 8;
+    table_clear_kernel<<<(unsigned)((n16 + 255) / 256), 256, 0, st>>>(x->at<Slot>(x->L.table), x->cfg.table_slots);
+    rc = launch_ok();
+    if (rc) return rc;
+    x->launches += 1;
+  }
+  if (M > 0) {
+    table_load_kernel<<<(unsigned)((M + 255) / 256), 256, 0, st>>>(x->at<Slot>(x->L.table), x->cfg.table_slots - 1, x->max_probe,
+                                                                   x->cfg.topk, dev_keys, dev_counts, dev_n_items, dev_ids,
+                                                                   dev_probs, M, x->at<unsigned long long>(x->L.stats));
+    rc = launch_ok();
+    if (rc == STAND_OK) x->launches += 1;
+  }
+  return rc;
+}
+
+int stand_state_dump(stand_ctx* x, int32_t* dev_tail, int64_t* dev_len, int32_t* dev_tree, int32_t* dev_cand_n,
+                     int32_t* dev_cand_id, float* dev_cand_phi, uint32_t* host_step, void* cu_stream) {
+  if (!x) return STAND_E_ARG;
+  cudaStream_t st = (cudaStream_t)cu_stream;
+  x->last_stream = st;
+  const stand_config& c = x->cfg;
+  const size_t BN = (size_t)c.B * c.N;
+  int rc = STAND_OK;
+  auto cp = [&](void* dst, size_t off, size_t bytes) {
+    if (rc == STAND_OK && dst) rc = cuda_ok(cudaMemcpyAsync(dst, x->ws + off, bytes, cudaMemcpyDeviceToDevice, st));
+  };
+  cp(dev_tail, x->L.tail, (size_t)c.B * c.order_max * 4);
+  cp(dev_len, x->L.len, (size_t)c.B * 8);
+  cp(dev_tree, x->L.tree, BN * 4);
+  cp(dev_cand_n, x->L.cand_n, BN * 4);
+  cp(dev_cand_id, x->L.cand_id, BN * c.topk * 4);
+  cp(dev_cand_phi, x->L.cand_phi, BN * c.topk * 4);
+  if (host_step) *host_step = x->step;
+  return rc;
+}
+
+int stand_state_load(stand_ctx* x, const int32_t* dev_tail, const int64_t* dev_len, const int32_t* dev_tree,
+                     const int32_t* dev_cand_n, const int32_t* dev_cand_id, const float* dev_cand_phi, uint32_t step,
+                     void* cu_stream) {
+  if (!x || !dev_tail || !dev_len || !dev_tree || !dev_cand_n || !dev_cand_id || !dev_cand_phi) return STAND_E_ARG;
+  cudaStream_t st = (cudaStream_t)cu_stream;
+  x->last_stream = st;
+  const stand_config& c = x->cfg;
+  const size_t BN = (size_t)c.B * c.N;
+  int rc = STAND_OK;
+  auto cp = [&](size_t off, const void* src, size_t bytes) {
+    if (rc == STAND_OK) rc = cuda_ok(cudaMemcpyAsync(x->ws + off, src, bytes, cudaMemcpyDeviceToDevice, st));
+  };
+  cp(x->L.tail, dev_tail, (size_t)c.B * c.order_max * 4);
+  cp(x->L.len, dev_len, (size_t)c.B * 8);
+  cp(x->L.tree, dev_tree, BN * 4);
+  cp(x->L.cand_n, dev_cand_n, BN * 4);
+  cp(x->L.cand_id, dev_cand_id, BN * c.topk * 4);
+  cp(x->L.cand_phi, dev_cand_phi, BN * c.topk * 4);
+  if (rc == STAND_OK) { x->step = step; x->pending = false; }
+  return rc;
+}
+
+uint64_t stand_launch_count(const stand_ctx* x) { return x ? x->launches : 0; }
+
+const char* stand_strerror(int code) {
+  switch (code) {
+    case STAND_OK: return "ok";
+    case STAND_E_ARG: return "invalid argument or configuration";
+    case STAND_E_WORKSPACE: return "workspace missing, misaligned or too small";
+    case STAND_E_CUDA: return "a CUDA runtime call failed";
+    case STAND_E_STATE: return "call not valid in the current state";
+    default: return "unknown error code";
+  }
+}
+
+}  // extern "C"

@@ -1,0 +1,129 @@
+"""Closed-loop comparison of the CUDA library with the CPU oracle on seeded synthetic workloads."""
+import numpy as np
+
+from oracle import stand_oracle as so
+from paper_2506_04708_b200 import inputs
+
+MARGIN_TOL = 1e-6  # a decision may differ from the oracle's only if the oracle logged a margin below this
+
+
+def value_tol(dtype):
+    """Relative tolerance of probabilities and stored values: 1e-5 for fp32 inputs, 4e-3 for bf16 inputs."""
+    return 1e-5 if dtype == inputs.DTYPE_F32 else 4e-3
+
+
+def to_device_logits(a, device="cuda:0"):
+    import torch
+    t = torch.from_numpy(a.view(np.int16) if a.dtype == np.uint16 else a)
+    t = t.to(device)
+    return t.view(torch.bfloat16) if a.dtype == np.uint16 else t
+
+
+def compare_tables(gpu_table, orc_table, tol, low_margin_keys=()):
+    """Returns a list of differences between two {key: (count, {id: prob})} maps."""
+    diffs = []
+    if set(gpu_table) != set(orc_table):
+        diffs.append(("keys", sorted(set(gpu_table) ^ set(orc_table))[:5]))
+        return diffs
+    for key, (cnt, items) in orc_table.items():
+        gcnt, gitems = gpu_table[key]
+        if gcnt != cnt:
+            diffs.append(("count", key, gcnt, cnt))
+            continue
+        if set(gitems) != set(items):
+            if key not in low_margin_keys:
+                diffs.append(("ids", key, sorted(gitems), sorted(items)))
+            continue
+        for t, pv in items.items():
+            if abs(gitems[t] - pv) > tol * abs(pv) + 1e-30:
+                diffs.append(("prob", key, t, gitems[t], pv))
+                break
+    return diffs
+
+
+def compare_states(gs, os_, tol):
+    diffs = []
+    for k in ("tail", "len", "tree", "cand_n", "step"):
+        if not np.array_equal(np.asarray(gs[k]), np.asarray(os_[k])):
+            diffs.append(k)
+    if "cand_n" not in diffs:
+        B, N = os_["cand_n"].shape
+        for b in range(B):
+            for u in range(N):
+                n = os_["cand_n"][b, u]
+                g = dict(zip(gs["cand_id"][b, u, :n].tolist(), gs["cand_phi"][b, u, :n].tolist()))
+                o = dict(zip(os_["cand_id"][b, u, :n].tolist(), os_["cand_phi"][b, u, :n].tolist()))
+                if set(g) != set(o) or any(abs(g[t] - o[t]) > tol * abs(o[t]) for t in o):
+                    diffs.append(("cand", b, u))
+    return diffs
+
+
+def resync_gpu_from_oracle(gpu, orc):
+    keys, counts, n_items, ids, probs = orc.table_arrays()
+    gpu.table_load(keys, counts, n_items, ids, probs.astype(np.float32), clear=True)
+    gpu.state_load(orc.state())
+
+
+class ClosedLoop:
+    """Runs the same seeded workload through both sides, step by step."""
+
+    def __init__(self, w, seed=0, peak_mode="add8", table_slots=None, prompt=8, device="cuda:0", **stand_kw):
+        from paper_2506_04708_b200.binding import Stand
+        self.w, self.seed, self.peak_mode = w, seed, peak_mode
+        self.parent = inputs.topology(w.N, w.D, w.kb)
+        self.depth = inputs.node_depths(self.parent)
+        self.streams = inputs.token_streams(w, seed, prompt + (w.steps + 2) * (w.D + 2))
+        slots = table_slots or w.table_slots
+        self.gpu = Stand(w.B, w.N, w.V, w.topk, w.order_max, w.dtype, w.T, seed, slots, self.parent, device=device,
+                         **stand_kw)
+        self.orc = so.Oracle(w.B, w.N, w.V, w.topk, w.order_max, w.dtype, w.T, seed, self.parent)
+        import torch
+        tail = np.full((w.B, w.order_max), -1, np.int32)
+        take = min(prompt, w.order_max)
+        tail[:, w.order_max - take:] = self.streams[:, prompt - take:prompt]
+        self.lens = np.full(w.B, prompt, np.int64)
+        self.gpu.reset_sequences(torch.from_numpy(tail), torch.from_numpy(self.lens))
+        self.orc.reset_sequences(tail, self.lens)
+        self.step_no = 0
+        self.tolerated = 0
+        self.emitted_total = 0
+        self.hard = []
+        self.low_margin_keys = set()
+
+    def step(self):
+        w = self.w
+        logits = inputs.logits_numpy(w, self.streams, self.lens, self.depth, self.step_no, self.seed, self.peak_mode)
+        dl = to_device_logits(logits, self.gpu.dev)
+        em_g, ne_g, tr_g = (t.cpu().numpy() for t in self.gpu.step(dl))
+        em_o, ne_o, tr_o = self.orc.step(logits)
+        ints, margins = self.orc.take_margins()
+        low = ints[margins < MARGIN_TOL]
+        for rec in low[low[:, 0] == so.MARGIN_MERGE]:
+            self.low_margin_keys.add(tuple(int(t) for t in rec[4:8] if t >= 0))
+        bad_b = set()
+        for b in range(w.B):
+            if ne_g[b] != ne_o[b] or not np.array_equal(em_g[b], em_o[b]) or not np.array_equal(tr_g[b], tr_o[b]):
+                bad_b.add(b)
+        if bad_b:
+            for b in sorted(bad_b):
+                excuse = low[(low[:, 1] == b) | (low[:, 0] == so.MARGIN_MERGE)]
+                if len(excuse) == 0:
+                    self.hard.append((self.step_no, b, em_g[b].tolist(), em_o[b].tolist(), tr_g[b].tolist(),
+                                      tr_o[b].tolist()))
+                else:
+                    self.tolerated += 1
+            resync_gpu_from_oracle(self.gpu, self.orc)
+        self.lens = self.orc.state()["len"]
+        self.emitted_total += int(ne_o.sum())
+        self.step_no += 1
+        return em_o, ne_o, tr_o
+
+    def check_state_and_table(self):
+        tol = value_tol(self.w.dtype)
+        d = compare_states(self.gpu.state_dump(), self.orc.state(), tol)
+        d += compare_tables(self.gpu.table_dict(), self.orc.table(), tol, self.low_margin_keys)
+        return d
+
+    def close(self):
+        self.gpu.close()
+        self.orc.close()

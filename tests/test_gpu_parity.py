@@ -1,0 +1,184 @@
+"""GPU parity: the CUDA library (through the C ABI) against the CPU oracle, element by element."""
+import numpy as np
+import pytest
+
+from oracle import stand_oracle as so
+from paper_2506_04708_b200 import inputs
+from tests import harness
+
+pytestmark = pytest.mark.gpu
+
+
+def _torch():
+    import torch
+    return torch
+
+
+# ------------------------------------------------------------------ row pass (a1)
+@pytest.mark.parametrize("dtype", ["f32", "bf16"])
+@pytest.mark.parametrize("V", [2, 13, 16, 1000, 1024, 1032, 5000, 32000, 151936])
+def test_row_stats_matches_oracle(dtype, V):
+    from paper_2506_04708_b200 import binding
+    torch = _torch()
+    rng = np.random.default_rng(V)
+    rows, k, T = 5, 10, 0.7
+    x = (rng.standard_normal((rows, V)) * 2.5).astype(np.float32)
+    x[0, rng.integers(0, V)] += 8
+    x[1, :] = np.round(x[1, :])          # many exact ties
+    x[2, :] = -30.0 - np.abs(x[2, :])    # far from zero: the offset logic must cope
+    if V > 1024:
+        x[3, :1024] -= 200.0             # first chunk far below the rest: forces a new offset
+        x[4] = np.sort(x[4])             # ascending: every vector brings new candidates
+    raw = inputs.f32_to_bf16_bits(x) if dtype == "bf16" else x
+    dl = harness.to_device_logits(raw)
+    lse, ids, vals, probs = (t.cpu().numpy() for t in binding.row_stats(dl, T, k))
+    tol = harness.value_tol(inputs.DTYPE_BF16 if dtype == "bf16" else inputs.DTYPE_F32)
+    for r in range(rows):
+        olse, oids, ovals, oprobs, _ = so.row_stats(raw[r], float(np.float32(T)), k)
+        assert np.array_equal(ids[r], oids), (r, ids[r], oids)
+        kk = min(k, V)
+        assert np.array_equal(vals[r, :kk].astype(np.float64), ovals[:kk])
+        assert abs(lse[r] - olse) <= 1e-5 * max(1.0, abs(olse))
+        assert np.allclose(probs[r, :kk], oprobs[:kk], rtol=tol, atol=1e-30)
+
+
+def test_row_stats_unaligned_rows_and_many_rows():
+    from paper_2506_04708_b200 import binding
+    torch = _torch()
+    rng = np.random.default_rng(5)
+    rows, V, k = 300, 1001, 8   # V*esize is not a multiple of 16: scalar loads
+    x = (rng.standard_normal((rows, V)) * 3).astype(np.float32)
+    for raw in (x, inputs.f32_to_bf16_bits(x)):
+        lse, ids, vals, probs = (t.cpu().numpy() for t in binding.row_stats(harness.to_device_logits(raw), 1.0, k))
+        for r in range(0, rows, 17):
+            olse, oids, ovals, oprobs, _ = so.row_stats(raw[r], 1.0, k)
+            assert np.array_equal(ids[r], oids)
+            assert abs(lse[r] - olse) <= 1e-5 * max(1.0, abs(olse))
+            assert np.allclose(probs[r], oprobs, rtol=1e-5 if raw.dtype == np.float32 else 4e-3)
+
+
+# ------------------------------------------------------------- whole step, closed loop
+def _run(w, steps, peak_mode, seed=0, check_every=0, **kw):
+    w = inputs.scaled(w, steps=steps)
+    loop = harness.ClosedLoop(w, seed=seed, peak_mode=peak_mode, **kw)
+    try:
+        for s in range(steps):
+            loop.step()
+            if check_every and (s + 1) % check_every == 0:
+                assert loop.check_state_and_table() == []
+        assert loop.hard == [], loop.hard[:3]
+        assert loop.check_state_and_table() == []
+        st = loop.gpu.stats()
+        assert st["drops"] == 0 and st["bad_tokens"] == 0
+        # a handful of low-margin decisions at most
+        assert loop.tolerated <= max(2, steps // 100)
+        return loop.emitted_total / (steps * w.B), loop.tolerated, st
+    finally:
+        loop.close()
+
+
+@pytest.mark.parametrize("peak_mode", ["add8", "p80"])
+def test_cfg1_full_run(peak_mode):
+    acc, tolerated, st = _run(inputs.WORKLOADS["cfg1"], 1000, peak_mode, table_slots=1 << 16, check_every=250)
+    if peak_mode == "p80":
+        assert acc > 1.5  # deep accept paths are exercised
+        assert sum(st["lookup_hits"]) > 0
+
+
+@pytest.mark.parametrize("peak_mode", ["add8", "p80"])
+def test_cfg2_window(peak_mode):
+    acc, _, st = _run(inputs.WORKLOADS["cfg2"], 48, peak_mode, table_slots=1 << 16, check_every=16)
+    if peak_mode == "p80":
+        assert acc > 1.5
+
+
+@pytest.mark.parametrize("peak_mode", ["add8", "p80"])
+def test_cfg3_window(peak_mode):
+    _run(inputs.WORKLOADS["cfg3"], 10, peak_mode, table_slots=1 << 16, check_every=5)
+
+
+def test_cfg4_window():
+    _run(inputs.WORKLOADS["cfg4"], 5, "p80", table_slots=1 << 16, check_every=5)
+
+
+def test_cfg5_shape_small_vocab():
+    # the tree-search shape (256 forked beams, shared prefixes -> many same-step updates of one context)
+    w = inputs.scaled(inputs.WORKLOADS["cfg5"], V=4096)
+    _run(w, 40, "p80", table_slots=1 << 18, check_every=10)
+
+
+@pytest.mark.parametrize("V,N,D,kb", [(16, 1, 0, 1), (13, 4, 2, 2), (50, 7, 3, 2), (1000, 16, 4, 3)])
+@pytest.mark.parametrize("dtype", [inputs.DTYPE_F32, inputs.DTYPE_BF16])
+def test_tiny_shapes(V, N, D, kb, dtype):
+    w = inputs.Workload("tiny", 3, N, D, kb, V, dtype, 0.9, 3, min(6, V), 60, 1 << 12, 2.0, 0.7, 12, 1.1)
+    _run(w, 60, "p80", check_every=20)
+
+
+# ------------------------------------------------------------------- stages on their own
+def test_stage_calls_equal_the_fused_step():
+    torch = _torch()
+    from paper_2506_04708_b200.binding import Stand
+    w = inputs.scaled(inputs.WORKLOADS["cfg1"], B=4, steps=30)
+    parent = inputs.topology(w.N, w.D, w.kb)
+    depth = inputs.node_depths(parent)
+    streams = inputs.token_streams(w, 3, 400)
+    a = Stand(w.B, w.N, w.V, w.topk, w.order_max, w.dtype, w.T, 3, 1 << 14, parent)
+    b = Stand(w.B, w.N, w.V, w.topk, w.order_max, w.dtype, w.T, 3, 1 << 14, parent)
+    tail = torch.from_numpy(streams[:, 5:8].copy())
+    lens = np.full(w.B, 8, np.int64)
+    a.reset_sequences(tail, torch.from_numpy(lens))
+    b.reset_sequences(tail, torch.from_numpy(lens))
+    for s in range(30):
+        dl = harness.to_device_logits(inputs.logits_numpy(w, streams, lens, depth, s, 3, "p80"))
+        ea, na, ta = (t.cpu().numpy().copy() for t in a.step(dl))
+        b.verify_tree(dl)
+        b.ngram_update()
+        b.draft_tree()
+        assert np.array_equal(ea, b.emitted.cpu().numpy()) and np.array_equal(na, b.n_emitted.cpu().numpy())
+        assert np.array_equal(ta, b.tree.cpu().numpy())
+        lens = a.state_dump()["len"]
+    assert a.table_dict() == b.table_dict()
+    # update without a pending verification is refused
+    from paper_2506_04708_b200.binding import StandError
+    with pytest.raises(StandError):
+        b.ngram_update()
+    a.close(); b.close()
+
+
+def test_bulk_update_and_table_roundtrip():
+    torch = _torch()
+    from paper_2506_04708_b200.binding import Stand
+    w = inputs.scaled(inputs.WORKLOADS["cfg5"], V=2000)
+    ctx, ids, probs = inputs.pregrow_records(w, 1, 6000)
+    parent = inputs.topology(w.N, w.D, w.kb)
+    g = Stand(1, w.N, w.V, w.topk, w.order_max, w.dtype, w.T, 0, 1 << 16, parent)
+    o = so.Oracle(1, w.N, w.V, w.topk, w.order_max, w.dtype, w.T, 0, parent)
+    g.ngram_update_bulk(torch.from_numpy(ctx), torch.from_numpy(ids), torch.from_numpy(probs))
+    o.update_bulk(ctx, ids, probs)
+    ot = o.table()
+    assert harness.compare_tables(g.table_dict(), ot, 1e-5) == []
+    assert g.stats()["inserts"] == len(ot) and g.stats()["drops"] == 0
+    # dump -> load into a fresh context -> same contents
+    g2 = Stand(1, w.N, w.V, w.topk, w.order_max, w.dtype, w.T, 0, 1 << 15, parent)
+    g2.table_load(*g.table_dump())
+    assert g2.table_dict() == g.table_dict()
+    g.close(); g2.close(); o.close()
+
+
+def test_full_table_drops_updates_and_never_hangs():
+    torch = _torch()
+    from paper_2506_04708_b200.binding import Stand
+    w = inputs.scaled(inputs.WORKLOADS["cfg5"], V=2000)
+    ctx, ids, probs = inputs.pregrow_records(w, 2, 3000)
+    parent = inputs.topology(w.N, w.D, w.kb)
+    g = Stand(1, w.N, w.V, w.topk, w.order_max, w.dtype, w.T, 0, 64, parent, max_probe=4)
+    g.ngram_update_bulk(torch.from_numpy(ctx), torch.from_numpy(ids), torch.from_numpy(probs))
+    st = g.stats()
+    assert st["drops"] > 0 and st["inserts"] <= 64
+    assert len(g.table_dict()) == st["inserts"]
+    g.close()
+
+
+def test_smoke_entry():
+    import __graft_entry__
+    __graft_entry__.smoke()
