@@ -192,8 +192,9 @@ def logits_numpy(w: Workload, streams, lens, depth, step: int, seed: int, peak_m
 
     Row (b, u) = sigma * N(0,1) noise with a planted peak at the stream token of
     the predicted position.  peak_mode "add8": +8 is added to that entry (the
-    contract reading).  "p80": the entry is set so that it holds 80% of the
-    row's mass before rounding (exercises deep accept paths and table hits).
+    contract reading).  "p80": the entry is set so that it holds 70-90% (80% on
+    average, varied per row) of the row's mass before rounding; this exercises deep
+    accept paths and table hits.
     """
     rng = np.random.default_rng([seed, 7_000_000 + step])
     x = rng.standard_normal((w.B, w.N, w.V), dtype=np.float32) * np.float32(w.sigma)
@@ -206,7 +207,8 @@ def logits_numpy(w: Workload, streams, lens, depth, step: int, seed: int, peak_m
         z[bb, uu, idx] = -np.inf
         m = z.max(axis=2, keepdims=True)
         lse = (m + np.log(np.exp(z - m).sum(axis=2, keepdims=True)))[:, :, 0]
-        x[bb, uu, idx] = (w.T * (math.log(4.0) + lse)).astype(np.float32)
+        mass = 0.7 + 0.2 * (((idx * 40503 + step * 9176 + uu * 131) % 1009) / 1009.0)  # 0.7 .. 0.9 per row
+        x[bb, uu, idx] = (w.T * (np.log(mass / (1.0 - mass)) + lse)).astype(np.float32)
     else:
         raise ValueError(peak_mode)
     for e in range(w.extra_peaks):
@@ -260,7 +262,9 @@ class DeviceLogits:
             z = rows.float() / w.T
             z[ar, flat] = float("-inf")
             lse = torch.logsumexp(z, dim=1)
-            rows[ar, flat] = (w.T * (math.log(4.0) + lse)).to(self.tdtype)
+            uu = ar % w.N
+            mass = 0.7 + 0.2 * (((flat * 40503 + step * 9176 + uu * 131) % 1009).double() / 1009.0)
+            rows[ar, flat] = (w.T * (torch.log(mass / (1.0 - mass)) + lse.double())).to(self.tdtype)
         for e in range(w.extra_peaks):
             h = (flat * 2654435761 + 97 * (e + 1) + step) % w.V
             on = ((flat + e + step) % 3) > e
