@@ -1,0 +1,348 @@
+#!/usr/bin/env python
+"""Benchmark of the STAND step (verify + N-gram update + draft) on synthetic workloads.
+
+    python bench.py [--gpus N] [--steps K] [--warmup W] [--workload cfg5] [--impl ours|reference]
+
+Prints ONE JSON line.  A step is one stand_step over one batch of logits [B, N, V].
+The timed region runs K steps back to back on one stream over a ring of pre-generated
+logit buffers that are resident in HBM (each step's input is far larger than L2 for the
+headline workload; smaller workloads use a ring that is larger than L2).
+"""
+import argparse
+import json
+import os
+import statistics
+import subprocess
+import sys
+import threading
+import time
+
+import numpy as np
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+if ROOT not in sys.path:
+    sys.path.insert(0, ROOT)
+
+from paper_2506_04708_b200 import inputs  # noqa: E402
+
+METRIC = "draft-tree nodes verified/sec at V=151,936 bf16"
+UNIT = "nodes/s"
+L2_BYTES = 126 * 2 ** 20
+
+
+def describe(w):
+    return (f"{w.name}: B={w.B} N={w.N} (depth {w.D}, <= {w.kb} children) V={w.V} "
+            f"{'bf16' if w.dtype == inputs.DTYPE_BF16 else 'fp32'} T={w.T} orders 1-{w.order_max} top-{w.topk} "
+            f"table {w.table_slots} slots")
+
+
+def measured_peaks():
+    path = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    if os.path.exists(path):
+        with open(path) as f:
+            return json.load(f), "measured"
+    return {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0}, "fallback"
+
+
+class ClockSampler:
+    """Samples nvidia-smi clocks and throttle reasons of one GPU while a region runs."""
+
+    Q = ("clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.hw_slowdown,"
+         "clocks_event_reasons.hw_thermal_slowdown,clocks_event_reasons.sw_thermal_slowdown,"
+         "clocks_event_reasons.sw_power_cap")
+
+    def __init__(self, index):
+        self.index, self.rows, self.proc = index, [], None
+
+    def start(self):
+        try:
+            self.proc = subprocess.Popen(["nvidia-smi", f"--query-gpu={self.Q}", "--format=csv,noheader,nounits",
+                                          "-i", str(self.index), "-lms", "100"], stdout=subprocess.PIPE, text=True)
+            self.t = threading.Thread(target=self._read, daemon=True)
+            self.t.start()
+        except Exception:
+            self.proc = None
+
+    def _read(self):
+        for line in self.proc.stdout:
+            self.rows.append([x.strip() for x in line.split(",")])
+
+    def stop(self):
+        if self.proc is None:
+            return {"sm_mhz": None, "sm_max_mhz": None, "reasons": ["nvidia-smi unavailable"]}
+        time.sleep(0.15)
+        self.proc.terminate()
+        self.t.join(timeout=2)
+        sm, mx, reasons = [], [], set()
+        for r in self.rows:
+            try:
+                sm.append(float(r[0])); mx.append(float(r[1]))
+            except Exception:
+                continue
+            for name, val in zip(("hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"), r[3:7]):
+                if val.lower().startswith("active"):
+                    reasons.add(name)
+        return {"sm_mhz": statistics.median(sm) if sm else None, "sm_max_mhz": max(mx) if mx else None,
+                "reasons": sorted(reasons), "samples": len(sm)}
+
+
+def physical_gpu_index(local):
+    vis = os.environ.get("CUDA_VISIBLE_DEVICES")
+    if vis:
+        try:
+            return int(vis.split(",")[local])
+        except Exception:
+            return local
+    return local
+
+
+def pregrow(gpu, w, seed, torch):
+    """Grows the table to about w.pregrow_contexts contexts with synthetic compressed rows."""
+    if not w.pregrow_contexts:
+        return 0
+    block, fed = 500_000, 0
+    for i in range(64):
+        if gpu.stats()["inserts"] >= 0.97 * w.pregrow_contexts:
+            break
+        ctx, ids, probs = inputs.pregrow_records(w, seed + 1000 * i, block)
+        gpu.ngram_update_bulk(torch.from_numpy(ctx), torch.from_numpy(ids), torch.from_numpy(probs))
+        fed += block
+    return gpu.stats()["inserts"]
+
+
+def run_ours(args, rank, world, local):
+    import torch
+    from paper_2506_04708_b200.binding import Stand
+
+    w = inputs.WORKLOADS[args.workload]
+    dev = torch.device("cuda", local)
+    torch.cuda.set_device(dev)
+    dist = None
+    if world > 1:
+        import torch.distributed as dist
+        dist.init_process_group("nccl", device_id=dev)
+    seed = args.seed + 7919 * rank  # every rank runs its own sequences: independent replicas
+    parent = inputs.topology(w.N, w.D, w.kb)
+    depth = inputs.node_depths(parent)
+    esize = 2 if w.dtype == inputs.DTYPE_BF16 else 4
+    step_bytes = w.B * w.N * w.V * esize
+    ring_n = max(4, min(16, int(40e9 // step_bytes)))
+    while ring_n * step_bytes < 3 * L2_BYTES:
+        ring_n += 1
+    ring_n = min(ring_n, 64)
+
+    gpu = Stand(w.B, w.N, w.V, w.topk, w.order_max, w.dtype, w.T, seed, w.table_slots, parent, device=dev,
+                host_staging=True)
+    contexts = pregrow(gpu, w, seed, torch)
+    prompt = 8
+    streams = inputs.token_streams(w, seed, prompt + (ring_n + 4) * (w.D + 2))
+    tail = np.full((w.B, w.order_max), -1, np.int32)
+    tail[:, :] = streams[:, prompt - w.order_max:prompt]
+    gpu.reset_sequences(torch.from_numpy(tail), torch.full((w.B,), prompt, dtype=torch.int64))
+
+    gen = inputs.DeviceLogits(w, streams, depth, seed, pool=2, device=dev, peak_mode=args.peak_mode)
+    tdtype = torch.bfloat16 if w.dtype == inputs.DTYPE_BF16 else torch.float32
+    ring = [torch.empty((w.B, w.N, w.V), dtype=tdtype, device=dev) for _ in range(ring_n)]
+    lens = torch.empty(w.B, dtype=torch.int64, device=dev)
+    # closed loop over the ring: every buffer gets its peaks at the positions its step predicts
+    for s in range(ring_n):
+        gpu.lens_device(lens)
+        gen.make(ring[s], lens, s)
+        gpu.step(ring[s])
+    del gen
+    torch.cuda.empty_cache()
+    for s in range(max(args.warmup, 3)):
+        gpu.step(ring[s % ring_n])
+    torch.cuda.synchronize()
+
+    def barrier():
+        if dist is not None:
+            dist.barrier()
+        torch.cuda.synchronize()
+
+    # ---- timed region: K steps back to back ------------------------------------------
+    sampler = ClockSampler(physical_gpu_index(local))
+    sampler.start()
+    time.sleep(0.25)
+    ev0, ev1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    launches0 = gpu.launch_count()
+    emitted0 = gpu.stats()["emitted_tokens"]
+    barrier()
+    torch.cuda.nvtx.range_push("stand_timed")
+    ev0.record()
+    for s in range(args.steps):
+        gpu.step(ring[s % ring_n])
+    ev1.record()
+    barrier()
+    torch.cuda.nvtx.range_pop()
+    ms_total = ev0.elapsed_time(ev1)
+    launches = gpu.launch_count() - launches0
+    st = gpu.stats()
+    accept_len = (st["emitted_tokens"] - emitted0) / (args.steps * w.B)
+
+    # ---- second pass: the row-pass kernel alone, timed by events around it -------------
+    n_prof = min(args.steps, 200)
+    evs = [(torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)) for _ in range(n_prof)]
+    for a, b in evs:  # torch creates the CUDA event at the first record; the library re-records it
+        a.record()
+        b.record()
+    for s in range(n_prof):
+        gpu.profile_row_pass(*evs[s])
+        gpu.step(ring[s % ring_n])
+    gpu.profile_row_pass(None, None)
+    torch.cuda.synchronize()
+    k1_ms = statistics.mean(a.elapsed_time(b) for a, b in evs)
+    clocks = sampler.stop()
+
+    if dist is not None:
+        t = torch.tensor([ms_total], dtype=torch.float64, device=dev)
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+        ms_total = float(t.item())
+    ms_per_step = ms_total / args.steps
+    nodes_per_step = w.B * w.N * world
+    value = nodes_per_step / (ms_per_step * 1e-3)
+
+    # ---- end to end through the C ABI with host buffers ---------------------------------
+    e2e_steps = max(2, min(8, int(4e9 // step_bytes) or 2))
+    h_logits = torch.empty((w.B, w.N, w.V), dtype=tdtype).pin_memory()
+    h_logits.copy_(ring[0])
+    h_em = torch.empty((w.B, gpu.D + 1), dtype=torch.int32).pin_memory()
+    h_ne = torch.empty(w.B, dtype=torch.int32).pin_memory()
+    h_tr = torch.empty((w.B, w.N), dtype=torch.int32).pin_memory()
+    gpu.step_host(h_logits, h_em, h_ne, h_tr)
+    barrier()
+    t0 = time.perf_counter()
+    for _ in range(e2e_steps):
+        gpu.step_host(h_logits, h_em, h_ne, h_tr)
+    barrier()
+    e2e_s = time.perf_counter() - t0
+    if dist is not None:
+        t = torch.tensor([e2e_s], dtype=torch.float64, device=dev)
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+        e2e_s = float(t.item())
+    e2e = {"value": nodes_per_step * e2e_steps / e2e_s, "unit": UNIT, "steps": e2e_steps,
+           "h2d_bytes_per_step": step_bytes, "d2h_bytes_per_step": (h_em.numel() + h_ne.numel() + h_tr.numel()) * 4}
+
+    peaks, peak_kind = measured_peaks()
+    alg_bytes = w.B * w.N * w.V * esize  # every logit is read once; everything else is < 1%
+    achieved = alg_bytes / (k1_ms * 1e-3) / 1e9
+    roofline = {"bound": "hbm", "kernel": "row_pass_kernel", "achieved": achieved, "peak": peaks["hbm_gbs"],
+                "unit": "GB/s", "frac": achieved / peaks["hbm_gbs"], "peak_kind": peak_kind + " copy bandwidth",
+                "traffic": None, "kernel_ms": k1_ms, "frac_of_nominal_8TBs": achieved / 8000.0,
+                "step_frac": alg_bytes / (ms_per_step * 1e-3) / 1e9 / peaks["hbm_gbs"]}
+    prof = os.path.join(ROOT, "profiles", f"traffic_{w.name}.json")
+    if os.path.exists(prof):
+        with open(prof) as f:
+            roofline["traffic"] = json.load(f).get("dram_bytes_per_launch")
+
+    cpu_baseline = None
+    if rank == 0 and world == 1 and not args.no_cpu_baseline:
+        cpu_baseline = time_oracle(w, ring[0], args, total_budget_s=12.0)
+
+    if rank == 0:
+        line = {
+            "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps,
+            "warmup": max(args.warmup, 3) + ring_n, "ms_per_step": ms_per_step, "higher_is_better": True,
+            "scaling": "weak", "vs_baseline": None, "dtype": "f32", "data": "synthetic",
+            "config": {"workload": describe(w), "peak_mode": args.peak_mode, "ring_buffers": ring_n,
+                       "l2": f"inputs larger than L2: {step_bytes / 1e6:.0f} MB per step, ring of {ring_n} "
+                             f"buffers = {ring_n * step_bytes / 1e9:.2f} GB",
+                       "table_contexts_at_start": int(contexts), "multi_gpu": "independent replicas per GPU"
+                       if world > 1 else "single GPU", "acceptance_length": accept_len},
+            "clocks": clocks, "e2e": e2e, "gpu_launches": int(launches), "roofline": roofline,
+            "logits_gbs": alg_bytes * world / (ms_per_step * 1e-3) / 1e9,
+            "table": {"drops": st["drops"], "max_probe": st["max_probe_seen"], "lookup_hits": st["lookup_hits"],
+                      "lookups": st["lookups"]},
+        }
+        if cpu_baseline is not None:
+            line["cpu_baseline"] = cpu_baseline
+        print(json.dumps(line))
+    gpu.close()
+    if dist is not None:
+        dist.destroy_process_group()
+
+
+def _oracle_inputs(w, ws, ring0, args, parent):
+    if ring0 is not None:
+        import torch
+        a = ring0[:ws.B].contiguous().cpu()
+        return a.view(torch.int16).numpy().view(np.uint16) if w.dtype == inputs.DTYPE_BF16 else a.numpy()
+    streams = inputs.token_streams(ws, args.seed, 64)
+    return inputs.logits_numpy(ws, streams, np.full(ws.B, 8), inputs.node_depths(parent), 0, args.seed, args.peak_mode)
+
+
+def _oracle_run(w, ws, logits, args, parent, n, warmup):
+    from oracle import stand_oracle as so
+    orc = so.Oracle(ws.B, w.N, w.V, w.topk, w.order_max, w.dtype, w.T, args.seed, parent)
+    orc.reset_sequences(np.full((ws.B, w.order_max), 5, np.int32), np.full(ws.B, 8, np.int64))
+    for _ in range(warmup):
+        orc.step(logits)
+    t0 = time.perf_counter()
+    for _ in range(n):
+        orc.step(logits)
+    dt = time.perf_counter() - t0
+    orc.take_margins()
+    orc.close()
+    return dt
+
+
+def time_oracle(w, ring0, args, total_budget_s, steps=None, warmup=0):
+    """Times the CPU oracle, as it stands, on a bounded sample of the workload: the first B_s sequences,
+    B_s chosen so that the whole run takes about total_budget_s on this machine's cores."""
+    cores = os.cpu_count() or 1
+    parent = inputs.topology(w.N, w.D, w.kb)
+    one = inputs.scaled(w, B=1)
+    t1 = _oracle_run(w, one, _oracle_inputs(w, one, ring0, args, parent), args, parent, 1, 0)  # one sequence, one step
+    if steps is None:
+        b = min(w.B, 2 * cores)
+        n = max(2, min(64, int(total_budget_s / (t1 * max(1.0, b / cores)))))
+    else:
+        n = steps
+        per_step = total_budget_s / max(1, steps + warmup)
+        b = max(1, min(w.B, int(per_step / t1) * cores if per_step >= t1 else 1))
+    ws = inputs.scaled(w, B=b)
+    dt = _oracle_run(w, ws, _oracle_inputs(w, ws, ring0, args, parent), args, parent, n, warmup)
+    return {"value": ws.B * w.N * n / dt, "unit": UNIT, "cores": cores, "kind": "oracle",
+            "sample": f"{n} steps of the first {ws.B} of {w.B} sequences ({ws.B * w.N} rows x V={w.V} per step), "
+                      f"table not pre-grown, OpenMP over sequences", "ms_per_step": dt / n * 1e3, "steps": n}
+
+
+def run_reference(args, rank, world):
+    """The oracle as it stands, on the host cores: the reference arm."""
+    if rank != 0:
+        return
+    w = inputs.WORKLOADS[args.workload]
+    r = time_oracle(w, None, args, total_budget_s=90.0, steps=args.steps, warmup=args.warmup)
+    line = {"impl": "reference", "metric": METRIC, "value": r["value"], "unit": UNIT, "n_gpus": world,
+            "steps": args.steps, "warmup": args.warmup, "ms_per_step": r["ms_per_step"], "higher_is_better": True,
+            "scaling": "weak", "vs_baseline": None, "dtype": "f64", "data": "synthetic",
+            "config": {"workload": describe(w), "peak_mode": args.peak_mode, "sample": r["sample"]},
+            "cpu_baseline": {"value": r["value"], "unit": UNIT, "cores": r["cores"], "kind": "oracle",
+                             "sample": r["sample"]},
+            "e2e": {"value": r["value"], "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+            "gpu_launches": 0}
+    print(json.dumps(line))
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=3000)
+    ap.add_argument("--warmup", type=int, default=20)
+    ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    ap.add_argument("--workload", default="cfg5", choices=sorted(inputs.WORKLOADS))
+    ap.add_argument("--peak-mode", default="add8", choices=["add8", "p80"])
+    ap.add_argument("--seed", type=int, default=0)
+    ap.add_argument("--no-cpu-baseline", action="store_true")
+    args = ap.parse_args()
+    rank = int(os.environ.get("RANK", "0"))
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    local = int(os.environ.get("LOCAL_RANK", "0"))
+    if args.impl == "reference":
+        run_reference(args, rank, world)
+    else:
+        run_ours(args, rank, world, local)
+
+
+if __name__ == "__main__":
+    main()

@@ -184,6 +184,11 @@ int stand_state_load(stand_ctx* ctx, const int32_t* dev_tail, const int64_t* dev
                      const int32_t* dev_cand_n, const int32_t* dev_cand_id, const float* dev_cand_phi,
                      uint32_t step, void* cu_stream);
 
+/* Timing hook for benchmarks: when both events (cudaEvent_t as void*) are non-NULL, every later
+ * verification records ev_before on the stream just before the row-pass kernel and ev_after just
+ * after it, so the caller can time that kernel alone.  NULL, NULL switches the hook off. */
+int stand_profile_row_pass(stand_ctx* ctx, void* ev_before, void* ev_after);
+
 /* How many kernels the library has launched through this context so far. */
 uint64_t stand_launch_count(const stand_ctx* ctx);
 

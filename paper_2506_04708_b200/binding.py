@@ -19,8 +19,8 @@ EXPORTS = [
     "stand_workspace_bytes", "stand_init", "stand_destroy", "stand_reset_sequences", "stand_verify_tree",
     "stand_ngram_update", "stand_ngram_update_bulk", "stand_draft_tree", "stand_step", "stand_step_host",
     "stand_row_stats_scratch_bytes", "stand_row_stats", "stand_get_stats", "stand_last_path", "stand_tree_depth",
-    "stand_table_dump", "stand_table_load", "stand_state_dump", "stand_state_load", "stand_launch_count",
-    "stand_strerror",
+    "stand_table_dump", "stand_table_load", "stand_state_dump", "stand_state_load", "stand_profile_row_pass",
+    "stand_launch_count", "stand_strerror",
 ]
 
 
@@ -80,6 +80,8 @@ def lib():
     L.stand_table_load.argtypes = [vp, vp, vp, vp, vp, vp, u64, i32, vp]
     L.stand_state_dump.argtypes = [vp, vp, vp, vp, vp, vp, vp, C.POINTER(u32), vp]
     L.stand_state_load.argtypes = [vp, vp, vp, vp, vp, vp, vp, u32, vp]
+    L.stand_profile_row_pass.argtypes = [vp, vp, vp]
+    L.stand_profile_row_pass.restype = C.c_int
     L.stand_launch_count.argtypes = [vp]
     L.stand_launch_count.restype = u64
     L.stand_strerror.argtypes = [C.c_int]
@@ -223,6 +225,18 @@ class Stand:
         _check(lib().stand_last_path(self.h, _ptr(path), _ptr(ids), _ptr(probs), _stream(None)), "stand_last_path")
         t.cuda.current_stream().synchronize()
         return path, ids, probs
+
+    def profile_row_pass(self, ev_before=None, ev_after=None):
+        """torch.cuda.Event pair (already created, enable_timing=True) recorded around the row-pass kernel."""
+        a = None if ev_before is None else C.c_void_p(ev_before.cuda_event)
+        b = None if ev_after is None else C.c_void_p(ev_after.cuda_event)
+        _check(lib().stand_profile_row_pass(self.h, a, b), "stand_profile_row_pass")
+
+    def lens_device(self, out):
+        """Copies the sequence lengths into `out` (int64 [B], device) on the current stream."""
+        _check(lib().stand_state_dump(self.h, None, _ptr(out), None, None, None, None, None, _stream(None)),
+               "stand_state_dump")
+        return out
 
     def launch_count(self):
         return lib().stand_launch_count(self.h)

@@ -118,6 +118,7 @@ struct stand_ctx {
   cudaStream_t last_stream;
   int max_probe;
   float c;  // log2(e) / T
+  cudaEvent_t ev_before, ev_after;  // optional timing hook around the row pass
 
   template <typename T> T* at(size_t off) const { return reinterpret_cast<T*>(ws + off); }
   int* topo_parent() const { return at<int>(L.topo); }
@@ -160,9 +161,11 @@ int launch_row_pass(const void* logits, long long rows, int V, int dtype, int n_
 
 int run_verify(stand_ctx* x, const void* logits, int32_t* emitted, int32_t* n_emitted, cudaStream_t st) {
   const stand_config& c = x->cfg;
+  if (x->ev_before) cudaEventRecord(x->ev_before, st);
   int rc = launch_row_pass(logits, (long long)c.B * c.N, c.V, c.dtype, x->d.n_chunks, x->d.cpu, x->d.upr, x->c, c.topk,
                            x->at<float2>(x->L.pairs), x->at<uint2>(x->L.part), st);
   if (rc) return rc;
+  if (x->ev_after) cudaEventRecord(x->ev_after, st);
   x->launches += 1;
   x->step += 1;  // the tree drafted in step s-1 is verified in step s
   VerifyParams v;
@@ -267,6 +270,8 @@ int stand_init(const stand_config* cfg, void* dev_workspace, size_t bytes, stand
   x->launches = 0;
   x->last_stream = 0;
   x->max_probe = cfg->max_probe > 0 ? cfg->max_probe : 128;
+  x->ev_before = nullptr;
+  x->ev_after = nullptr;
   x->c = log2e_over_T(cfg->temperature);
 
   int topo[4 * NODES_MAX + DEPTH_MAX + 2];
@@ -536,6 +541,13 @@ int stand_state_load(stand_ctx* x, const int32_t* dev_tail, const int64_t* dev_l
   cp(x->L.cand_phi, dev_cand_phi, BN * c.topk * 4);
   if (rc == STAND_OK) { x->step = step; x->pending = false; }
   return rc;
+}
+
+int stand_profile_row_pass(stand_ctx* x, void* ev_before, void* ev_after) {
+  if (!x || ((ev_before == nullptr) != (ev_after == nullptr))) return STAND_E_ARG;
+  x->ev_before = (cudaEvent_t)ev_before;
+  x->ev_after = (cudaEvent_t)ev_after;
+  return STAND_OK;
 }
 
 uint64_t stand_launch_count(const stand_ctx* x) { return x ? x->launches : 0; }
