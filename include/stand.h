@@ -63,7 +63,7 @@ typedef struct {
   int32_t order_max;   /* N-gram orders 1..order_max, <= STAND_MAX_ORDER */
   int32_t dtype;       /* STAND_DTYPE_* of the logits */
   float temperature;   /* > 0 (Sec. 5: all sampling at temperature T) */
-  int32_t max_probe;   /* hash-table probe limit, >= 1 (0 = default 128) */
+  int32_t max_probe;   /* hash-table probe limit, >= 1 (0 = default 96) */
   uint64_t seed;
   uint64_t table_slots;   /* power of two, >= 2; one slot = 128 bytes */
   const int32_t* parent;  /* HOST, [N]; parent[0] = -1; read during stand_init only */

@@ -1,7 +1,7 @@
 // Stochastic tree drafting (paper Sec. 4.2).  One thread block per sequence walks
 // the static topology level by level; one warp per parent node:
 //   - the contexts of order n_max..1 of the would-be sequence (tail + path tokens)
-//     are probed at once, one lane per order; the longest hit wins ("first
+//     are probed at once, 8 lanes per order; the longest hit wins ("first
 //     successful match", longest first);
 //   - the hit's candidates (id, phi) sit one per lane; Gumbel-Top-K: each lane
 //     forms g = log(phi) - log(-log U) with its own Philox uniform (keyed by the
@@ -59,27 +59,30 @@ __global__ void __launch_bounds__(K4_THREADS) draft_kernel(const DraftParams p) 
         while (w != 0 && filled < n_max) { win[n_max - 1 - filled] = s_tok[w]; ++filled; w = p.parent[w]; }
         for (int i = n_max - 1; filled < n_max; --i, ++filled) win[n_max - 1 - filled] = p.tail[b * n_max + i];
       }
-      // one lane per order
-      uint32_t slot = NO_SLOT;
-      if (lane < n_max) {
-        const int n = lane + 1;
-        int key[4] = {-1, -1, -1, -1};
-        bool ok = true;
+      // one group of 8 lanes per order: all orders are probed at once
+      const int grp = lane / GROUP;
+      int key[4] = {-1, -1, -1, -1};
+      bool ok = grp < n_max;
+      if (ok) {
+        const int n = grp + 1;
         for (int i = 0; i < n; ++i) {
           const int t = win[n_max - n + i];
           if (t < 0 || t >= p.V) ok = false;
           key[4 - n + i] = t;
         }
-        if (ok) slot = find_slot(p.table, p.mask, p.max_probe, key);
       }
-      const unsigned hits = __ballot_sync(FULL, slot != NO_SLOT);
+      uint32_t slot = find_slot_group(p.table, p.mask, p.max_probe, key, ok);
+      const unsigned found = __ballot_sync(FULL, slot != NO_SLOT);
+      unsigned hits = 0;  // bit n-1: order n matched
+      for (int gq = 0; gq < 32 / GROUP; ++gq)
+        if ((found >> (gq * GROUP)) & 1u) hits |= 1u << gq;
       if (lane == 0) {
         atomicAdd(&p.stats[ST_LOOKUPS], 1ull);
         if (hits) atomicAdd(&p.stats[ST_HIT0 + (31 - __clz(hits))], 1ull);
       }
       if (hits == 0) { if (lane == 0) p.cand_n[row] = 0; continue; }
       const int winner = 31 - __clz(hits);  // the longest order that matched
-      slot = __shfl_sync(FULL, slot, winner);
+      slot = __shfl_sync(FULL, slot, winner * GROUP);
       const Slot* s = &p.table[slot];
       const int n_items = (int)s->n_items;
       int id = -1;

@@ -17,7 +17,7 @@ using namespace stand;
 
 namespace {
 
-constexpr int BULK_ROWS = 2048;  // rows per batch of the bulk update
+constexpr int BULK_ROWS = 16384;  // rows per batch of the bulk update
 
 struct Layout {
   size_t table, topo, tail, len, tree, cand_n, cand_id, cand_phi, pairs, part, emitted, n_path, path, rec_ctx, rec_ids,
@@ -195,11 +195,10 @@ int run_update_rows(stand_ctx* x, long long n_rows, const int* ctxw, const int* 
   u.n_max = c.order_max; u.n_rows = n_rows; u.rec_ctx = ctxw; u.rec_ids = ids; u.rec_p = probs; u.n_path = n_path;
   u.width = width; u.rec_slot = x->at<uint32_t>(x->L.rec_slot); u.stats = x->at<unsigned long long>(x->L.stats);
   const long long n_rec = n_rows * c.order_max;
-  const unsigned blocks = (unsigned)((n_rec + 255) / 256);
-  update_locate_kernel<<<blocks, 256, 0, st>>>(u);
+  update_locate_kernel<<<(unsigned)((n_rec * GROUP + 255) / 256), 256, 0, st>>>(u);
   int rc = launch_ok();
   if (rc) return rc;
-  update_apply_kernel<<<blocks, 256, 0, st>>>(u);
+  update_apply_kernel<<<(unsigned)((n_rec + APPLY_WARPS - 1) / APPLY_WARPS), APPLY_WARPS * 32, 0, st>>>(u);
   rc = launch_ok();
   if (rc) return rc;
   x->launches += 2;
@@ -269,7 +268,7 @@ int stand_init(const stand_config* cfg, void* dev_workspace, size_t bytes, stand
   x->pending = false;
   x->launches = 0;
   x->last_stream = 0;
-  x->max_probe = cfg->max_probe > 0 ? cfg->max_probe : 128;
+  x->max_probe = cfg->max_probe > 0 ? cfg->max_probe : 96;
   x->ev_before = nullptr;
   x->ev_after = nullptr;
   x->c = log2e_over_T(cfg->temperature);
@@ -491,7 +490,7 @@ int stand_table_load(stand_ctx* x, const int32_t* dev_keys, const uint32_t* dev_
     x->launches += 1;
   }
   if (M > 0) {
-    table_load_kernel<<<(unsigned)((M + 255) / 256), 256, 0, st>>>(x->at<Slot>(x->L.table), x->cfg.table_slots - 1, x->max_probe,
+    table_load_kernel<<<(unsigned)((M * GROUP + 255) / 256), 256, 0, st>>>(x->at<Slot>(x->L.table), x->cfg.table_slots - 1, x->max_probe,
                                                                    x->cfg.topk, dev_keys, dev_counts, dev_n_items, dev_ids,
                                                                    dev_probs, M, x->at<unsigned long long>(x->L.stats));
     rc = launch_ok();

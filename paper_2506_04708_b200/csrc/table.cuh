@@ -2,22 +2,33 @@
 // device memory.  A slot is one 128-byte line: the context (up to 4 tokens, -1
 // padded at the front, so the order is the number of tokens), the number of
 // distributions averaged so far, and up to 12 (token id, mean probability) pairs.
-// A context is claimed lock-free with a single 16-byte compare-and-swap on the key.
+//
+// Probing: double hashing (odd stride over a power-of-two table), so probe
+// lengths stay short at high load and do not cluster.  A lookup is made by a
+// group of 8 lanes that read 8 probe positions at once: nearly every lookup costs
+// one memory round trip.  A context is claimed lock-free with a single 16-byte
+// compare-and-swap on the key; entries are never removed, so a key lives at the
+// first position of its probe sequence that was free when it arrived.
 //
 // "Efficient logit approximation": a repeat of a context seen c times is merged as
 // old * c/(c+1) + new * 1/(c+1) over the union of ids (missing = 0) and cut to the
 // top-k again.  The merge is not commutative, so same-step updates of one context
-// are applied in record order by the record with the lowest index.
+// are applied in record order: stage 1 notes per slot the lowest record that maps
+// to it and how many do; in stage 2 the warp of that record applies them all.
 #pragma once
 #include "common.cuh"
 
 namespace stand {
 
+constexpr int GROUP = 8;               // lanes that probe together
+constexpr uint32_t NO_REC = 0xFFFFFFFFu;
+
 struct __align__(128) Slot {
   int key[4];         // -1,-1,-1,-1 = empty
   uint32_t count;     // distributions averaged
   uint32_t n_items;   // stored pairs
-  uint32_t pad[2];
+  uint32_t lead;      // during an update: lowest row whose record maps here; NO_REC otherwise
+  uint32_t pend;      // during an update: how many records map here; 0 otherwise
   int ids[KMAX];
   float probs[KMAX];
 };
@@ -36,6 +47,20 @@ __device__ __forceinline__ unsigned long long hash_key(const int (&k)[4]) {
   return h;
 }
 
+// Probe i of a key sits at (start + i * stride) & mask; stride is odd, so the
+// sequence visits every slot of a power-of-two table.
+struct ProbeSeq {
+  unsigned long long start, stride;
+};
+__device__ __forceinline__ ProbeSeq probe_seq(const int (&key)[4], unsigned long long mask) {
+  const unsigned long long h = hash_key(key);
+  ProbeSeq p;
+  p.start = h & mask;
+  p.stride = ((h >> 40) | 1ull) & mask;
+  if (p.stride == 0) p.stride = 1;
+  return p;
+}
+
 __device__ __forceinline__ ulonglong2 cas128(void* addr, ulonglong2 expected, ulonglong2 desired) {
   ulonglong2 old;
   asm volatile(
@@ -50,6 +75,19 @@ __device__ __forceinline__ ulonglong2 cas128(void* addr, ulonglong2 expected, ul
   return old;
 }
 
+// One 16-byte key read as a single access, safe against a concurrent cas128.
+__device__ __forceinline__ ulonglong2 ld_key_relaxed(const void* addr) {
+  ulonglong2 v;
+  asm volatile(
+      "{\n\t.reg .b128 t;\n\t"
+      "ld.relaxed.gpu.global.b128 t, [%2];\n\t"
+      "mov.b128 {%0, %1}, t;\n\t}"
+      : "=l"(v.x), "=l"(v.y)
+      : "l"(addr)
+      : "memory");
+  return v;
+}
+
 __device__ __forceinline__ ulonglong2 pack_key(const int (&k)[4]) {
   ulonglong2 r;
   r.x = (unsigned long long)(uint32_t)k[0] | ((unsigned long long)(uint32_t)k[1] << 32);
@@ -57,37 +95,91 @@ __device__ __forceinline__ ulonglong2 pack_key(const int (&k)[4]) {
   return r;
 }
 
-// Finds the slot of `key`, claiming an empty one if the key is new.  Bounded
-// linear probing; NO_SLOT when the limit is reached.
-__device__ __forceinline__ uint32_t find_or_insert(Slot* table, unsigned long long mask, int max_probe,
-                                                   const int (&key)[4], unsigned long long* stats) {
+// Finds the slot of `key`, claiming a free one if the key is new.  Called by ALL 32
+// lanes of a warp; the 8 lanes of a group share one key (`live` false: the group
+// has no work and only takes part in the votes).  Bounded: at most max_probe
+// positions are tried, then the update is dropped and NO_SLOT returned.
+__device__ __forceinline__ uint32_t find_or_insert_group(Slot* table, unsigned long long mask, int max_probe,
+                                                         const int (&key)[4], bool live, unsigned long long* stats) {
+  const int lane = threadIdx.x & 31, gl = lane & (GROUP - 1), gbase = lane & ~(GROUP - 1);
   const ulonglong2 mine = pack_key(key);
   const ulonglong2 empty = make_ulonglong2(~0ull, ~0ull);
-  unsigned long long h = hash_key(key);
-  for (int i = 0; i < max_probe; ++i) {
-    const unsigned long long s = (h + (unsigned long long)i) & mask;
-    const ulonglong2 old = cas128(&table[s], empty, mine);
-    const bool claimed = old.x == empty.x && old.y == empty.y;
-    if (claimed || (old.x == mine.x && old.y == mine.y)) {
-      if (i > 0) atomicMax(&stats[ST_MAX_PROBE], (unsigned long long)i);
-      return (uint32_t)s;
+  const ProbeSeq ps = probe_seq(key, mask);
+  uint32_t result = NO_SLOT;
+  bool done = !live;
+  for (int base = 0; __any_sync(FULL, !done); base += GROUP) {
+    if (!done && base >= max_probe) {
+      done = true;
+      if (gl == 0) atomicAdd(&stats[ST_DROPS], 1ull);
+    }
+    const int i = base + gl;
+    const unsigned long long s = (ps.start + (unsigned long long)i * ps.stride) & mask;
+    int st = 0;  // 0: another key, 1: this key, 2: free
+    if (!done && i < max_probe) {
+      const ulonglong2 k = ld_key_relaxed(&table[s]);
+      st = (k.x == mine.x && k.y == mine.y) ? 1 : ((k.x == empty.x && k.y == empty.y) ? 2 : 0);
+    }
+    // settle the positions of this batch in probe order
+    for (;;) {
+      const unsigned votes = __ballot_sync(FULL, !done && st != 0);
+      const unsigned mine_votes = (votes >> gbase) & ((1u << GROUP) - 1u);
+      const bool active = !done && mine_votes != 0;
+      if (!__any_sync(FULL, active)) break;
+      const int first = mine_votes ? __ffs(mine_votes) - 1 : 0;
+      int outcome = 0;  // 1: settled at this position, 2: lost the position to another key
+      if (active && gl == first) {
+        if (st == 1) outcome = 1;
+        else {
+          const ulonglong2 old = cas128(&table[s], empty, mine);
+          const bool ok = (old.x == empty.x && old.y == empty.y) || (old.x == mine.x && old.y == mine.y);
+          outcome = ok ? 1 : 2;
+        }
+      }
+      outcome = __shfl_sync(FULL, outcome, gbase + first);
+      const unsigned long long s_first = __shfl_sync(FULL, s, gbase + first);
+      if (active) {
+        if (outcome == 1) {
+          result = (uint32_t)s_first;
+          done = true;
+          if (gl == 0 && base + first > 0) atomicMax(&stats[ST_MAX_PROBE], (unsigned long long)(base + first));
+        } else if (gl == first) {
+          st = 0;
+        }
+      }
     }
   }
-  atomicAdd(&stats[ST_DROPS], 1ull);
-  return NO_SLOT;
+  return result;
 }
 
-// Read-only lookup (no writer may be active).
-__device__ __forceinline__ uint32_t find_slot(const Slot* table, unsigned long long mask, int max_probe,
-                                              const int (&key)[4]) {
-  unsigned long long h = hash_key(key);
-  for (int i = 0; i < max_probe; ++i) {
-    const unsigned long long s = (h + (unsigned long long)i) & mask;
-    const int4 k = *reinterpret_cast<const int4*>(table[s].key);
-    if (k.x == key[0] && k.y == key[1] && k.z == key[2] && k.w == key[3]) return (uint32_t)s;
-    if (k.x == -1 && k.y == -1 && k.z == -1 && k.w == -1) return NO_SLOT;
+// Read-only lookup by a group of 8 lanes (no writer may be active).  Called by ALL
+// 32 lanes of a warp, as above.
+__device__ __forceinline__ uint32_t find_slot_group(const Slot* table, unsigned long long mask, int max_probe,
+                                                    const int (&key)[4], bool live) {
+  const int lane = threadIdx.x & 31, gl = lane & (GROUP - 1), gbase = lane & ~(GROUP - 1);
+  const ProbeSeq ps = probe_seq(key, mask);
+  uint32_t result = NO_SLOT;
+  bool done = !live;
+  for (int base = 0; __any_sync(FULL, !done); base += GROUP) {
+    if (base >= max_probe) done = true;
+    const int i = base + gl;
+    const unsigned long long s = (ps.start + (unsigned long long)i * ps.stride) & mask;
+    int st = 0;
+    if (!done && i < max_probe) {
+      const int4 k = *reinterpret_cast<const int4*>(table[s].key);
+      st = (k.x == key[0] && k.y == key[1] && k.z == key[2] && k.w == key[3]) ? 1
+           : ((k.x == -1 && k.y == -1 && k.z == -1 && k.w == -1) ? 2 : 0);
+    }
+    const unsigned votes = __ballot_sync(FULL, !done && st != 0);
+    const unsigned mine_votes = (votes >> gbase) & ((1u << GROUP) - 1u);
+    const int first = mine_votes ? __ffs(mine_votes) - 1 : 0;
+    const int st_first = __shfl_sync(FULL, st, gbase + first);
+    const unsigned long long s_first = __shfl_sync(FULL, s, gbase + first);
+    if (!done && mine_votes != 0) {
+      if (st_first == 1) result = (uint32_t)s_first;
+      done = true;  // the key, or a free position before it: absent
+    }
   }
-  return NO_SLOT;
+  return result;
 }
 
 __global__ void table_clear_kernel(Slot* table, unsigned long long n_slots) {
@@ -95,13 +187,16 @@ __global__ void table_clear_kernel(Slot* table, unsigned long long n_slots) {
   const unsigned long long i = (unsigned long long)blockIdx.x * blockDim.x + threadIdx.x;
   if (i >= n_slots * 8) return;
   uint4* w = reinterpret_cast<uint4*>(table) + i;
-  *w = (i & 7) == 0 ? make_uint4(~0u, ~0u, ~0u, ~0u) : make_uint4(0u, 0u, 0u, 0u);
+  const int part = (int)(i & 7);
+  *w = part == 0 ? make_uint4(~0u, ~0u, ~0u, ~0u) : (part == 1 ? make_uint4(0u, 0u, NO_REC, 0u) : make_uint4(0u, 0u, 0u, 0u));
 }
 
 // ---------------------------------------------------------------------------
-// Update, stage 1: record r = (row, order n) -> slot.  Rows are compressed
+// Update, stage 1: record (row, order n) -> slot.  Rows are compressed
 // distributions with a context window of n_max tokens; for the step path row =
 // (sequence, path position) and only the first n_path[sequence] positions count.
+// One group of 8 lanes per record.  rec_slot is laid out [n_max][n_rows], so the
+// records that can share a slot (same order) are contiguous.
 // ---------------------------------------------------------------------------
 struct UpdateParams {
   Slot* table;
@@ -113,94 +208,144 @@ struct UpdateParams {
   const float* rec_p;   // [n_rows, K]
   const int* n_path;    // [n_rows / width] or null (all rows count)
   int width;            // rows per sequence when n_path is given
-  uint32_t* rec_slot;   // [n_rows * n_max]
+  uint32_t* rec_slot;   // [n_max, n_rows]
   unsigned long long* stats;
 };
 
-__global__ void __launch_bounds__(256) update_locate_kernel(const UpdateParams p) {
-  const long long r = (long long)blockIdx.x * blockDim.x + threadIdx.x;
-  if (r >= p.n_rows * p.n_max) return;
-  const long long row = r / p.n_max;
-  const int n = (int)(r - row * p.n_max) + 1;
-  uint32_t slot = NO_SLOT;
-  bool live = true;
-  if (p.n_path) live = (int)(row % p.width) < p.n_path[row / p.width];
-  if (live) {
-    int key[4] = {-1, -1, -1, -1};
-    bool ok = true;
+// The locate step of one record; called by all lanes of a warp, 8 lanes per record.
+__device__ __forceinline__ void locate_record(const UpdateParams& p, long long row, int n, bool in_range) {
+  const int gl = threadIdx.x & (GROUP - 1);
+  int key[4] = {-1, -1, -1, -1};
+  bool ok = in_range;
+  if (ok && p.n_path) ok = (int)(row % p.width) < p.n_path[row / p.width];
+  if (ok) {
     for (int i = 0; i < n; ++i) {
       const int t = p.rec_ctx[row * p.n_max + (p.n_max - n + i)];
-      if (t < 0) ok = false;           // context shorter than n: this order is skipped
-      else if (t >= p.V) { ok = false; atomicAdd(&p.stats[ST_BAD_TOKENS], 1ull); }
+      if (t < 0) ok = false;  // context shorter than n: this order is skipped
+      else if (t >= p.V) {
+        ok = false;
+        if (gl == 0) atomicAdd(&p.stats[ST_BAD_TOKENS], 1ull);
+      }
       key[4 - n + i] = t;
     }
-    if (ok) slot = find_or_insert(p.table, p.mask, p.max_probe, key, p.stats);
   }
-  p.rec_slot[r] = slot;
+  const uint32_t slot = find_or_insert_group(p.table, p.mask, p.max_probe, key, ok, p.stats);
+  if (in_range && gl == 0) {
+    p.rec_slot[(long long)(n - 1) * p.n_rows + row] = slot;
+    if (slot != NO_SLOT) {
+      atomicMin(&p.table[slot].lead, (uint32_t)row);
+      atomicAdd(&p.table[slot].pend, 1u);
+    }
+  }
 }
 
-// One merge of a compressed row into a slot image held in registers/local memory.
-__device__ __forceinline__ void merge_into(int (&ids)[KMAX], float (&probs)[KMAX], uint32_t& count, uint32_t& n_items,
-                                           const int* f_ids, const float* f_p, int K) {
-  int mid[2 * KMAX];
-  double mval[2 * KMAX];
-  int n = 0;
-  const double c = (double)count;
-  const double w_old = c / (c + 1.0), w_new = 1.0 / (c + 1.0);
-  for (uint32_t i = 0; i < n_items; ++i) { mid[n] = ids[i]; mval[n] = __dmul_rn((double)probs[i], w_old); ++n; }
-  for (int i = 0; i < K; ++i) {
-    const int id = f_ids[i];
-    if (id < 0) continue;
-    const double add = __dmul_rn((double)f_p[i], w_new);
-    int at = -1;
-    for (int j = 0; j < n; ++j)
-      if (mid[j] == id) at = j;
-    if (at >= 0) mval[at] = __dadd_rn(mval[at], add);
-    else { mid[n] = id; mval[n] = add; ++n; }
-  }
-  // the k most probable, equal probabilities by lower id
-  const int keep = n < K ? n : K;
-  for (int r = 0; r < keep; ++r) {
-    int best = r;
-    for (int j = r + 1; j < n; ++j)
-      if (mval[j] > mval[best] || (mval[j] == mval[best] && mid[j] < mid[best])) best = j;
-    const int ti = mid[r]; mid[r] = mid[best]; mid[best] = ti;
-    const double tv = mval[r]; mval[r] = mval[best]; mval[best] = tv;
-    ids[r] = mid[r];
-    probs[r] = (float)mval[r];
-  }
-  n_items = (uint32_t)keep;
-  count += 1;
+__global__ void __launch_bounds__(256) update_locate_kernel(const UpdateParams p) {
+  const long long g = ((long long)blockIdx.x * blockDim.x + threadIdx.x) / GROUP;  // record index
+  const bool in_range = g < p.n_rows * p.n_max;
+  const long long row = in_range ? g / p.n_max : 0;
+  const int n = in_range ? (int)(g - row * p.n_max) + 1 : 1;
+  locate_record(p, row, n, in_range);
 }
 
-// Update, stage 2: the lowest-index record of every slot applies all records of
-// that slot in index order (the canonical order of same-step updates).
-__global__ void __launch_bounds__(256) update_apply_kernel(const UpdateParams p) {
-  const long long n_rec = p.n_rows * p.n_max;
-  const long long r = (long long)blockIdx.x * blockDim.x + threadIdx.x;
-  if (r >= n_rec) return;
-  const uint32_t slot = p.rec_slot[r];
-  if (slot == NO_SLOT) return;
-  for (long long i = 0; i < r; ++i)
-    if (__ldg(&p.rec_slot[i]) == slot) return;  // an earlier record leads this slot
-  Slot* s = &p.table[slot];
+// ---------------------------------------------------------------------------
+// One merge of a compressed row into a slot image in shared memory, by a whole
+// warp.  Lanes 0..11 carry the stored pairs, lanes 16..27 the fresh ones; equal
+// ids are paired with match_any, every lane ranks its pair among all of them by
+// (probability descending, id ascending), and the K best are written back.
+// ---------------------------------------------------------------------------
+struct SlotImage {
+  uint32_t count, n_items;
   int ids[KMAX];
   float probs[KMAX];
-  uint32_t count = s->count, n_items = s->n_items;
-  for (int i = 0; i < KMAX; ++i) { ids[i] = s->ids[i]; probs[i] = s->probs[i]; }
-  const bool fresh_slot = count == 0;
-  unsigned long long applied = 0;
-  for (long long i = r; i < n_rec; ++i) {
-    if (i != r && __ldg(&p.rec_slot[i]) != slot) continue;
-    const long long row = i / p.n_max;
-    merge_into(ids, probs, count, n_items, p.rec_ids + row * p.K, p.rec_p + row * p.K, p.K);
-    ++applied;
+};
+
+__device__ __forceinline__ void merge_warp(SlotImage* img, const int* f_ids, const float* f_p, int K, int lane) {
+  const double c = (double)img->count;
+  const double w_old = c / (c + 1.0), w_new = 1.0 / (c + 1.0);
+  const int n_items = (int)img->n_items;
+  int id = -2 - lane;  // lanes without a pair carry distinct negative ids
+  double val = 0.0;
+  bool valid = false;
+  if (lane < KMAX) {
+    if (lane < n_items) { id = img->ids[lane]; val = __dmul_rn((double)img->probs[lane], w_old); valid = true; }
+  } else if (lane >= 16 && lane < 16 + K) {
+    const int fid = f_ids[lane - 16];
+    if (fid >= 0) { id = fid; val = __dmul_rn((double)f_p[lane - 16], w_new); valid = true; }
   }
-  s->count = count;
-  s->n_items = n_items;
-  for (int i = 0; i < KMAX; ++i) { s->ids[i] = i < (int)n_items ? ids[i] : 0; s->probs[i] = i < (int)n_items ? probs[i] : 0.0f; }
-  atomicAdd(&p.stats[ST_RECORDS], applied);
-  if (fresh_slot) atomicAdd(&p.stats[ST_INSERTS], 1ull);
+  // pair a fresh id with the same stored id
+  const unsigned same = __match_any_sync(FULL, id);
+  const unsigned other = same & ~(1u << lane);
+  const int partner = other ? __ffs(other) - 1 : lane;
+  const double pval = __shfl_sync(FULL, val, partner);
+  if (valid && other) {
+    if (lane < 16) val = __dadd_rn(val, pval);  // the stored pair absorbs the fresh one
+    else valid = false;
+  }
+  __syncwarp();
+  int rank = 0;
+  for (int j = 0; j < 16 + KMAX; ++j) {
+    if (j == KMAX) j = 16;
+    const double vj = __shfl_sync(FULL, val, j);
+    const int idj = __shfl_sync(FULL, id, j);
+    const bool okj = __shfl_sync(FULL, (int)valid, j) != 0;
+    if (okj && (vj > val || (vj == val && idj < id))) ++rank;
+  }
+  const int n_valid = __popc(__ballot_sync(FULL, valid));
+  __syncwarp();
+  if (valid && rank < K) { img->ids[rank] = id; img->probs[rank] = (float)val; }
+  if (lane == 0) { img->n_items = (uint32_t)(n_valid < K ? n_valid : K); img->count += 1; }
+  __syncwarp();
+}
+
+// Update, stage 2: one warp per record.  The warp of the lowest row of a slot
+// applies all records of that slot in row order (the canonical order of same-step
+// updates) and closes the slot's update fields.
+constexpr int APPLY_WARPS = 8;
+__global__ void __launch_bounds__(APPLY_WARPS * 32) update_apply_kernel(const UpdateParams p) {
+  __shared__ SlotImage s_img[APPLY_WARPS];
+  const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+  const long long g = (long long)blockIdx.x * APPLY_WARPS + warp;
+  if (g >= p.n_rows * p.n_max) return;
+  // order-major, so that the warps of a block work on neighbouring rows of one order
+  const int n = (int)(g / p.n_rows) + 1;
+  const long long row = g - (long long)(n - 1) * p.n_rows;
+  const uint32_t* seg = p.rec_slot + (long long)(n - 1) * p.n_rows;
+  const uint32_t slot = seg[row];
+  if (slot == NO_SLOT) return;
+  Slot* s = &p.table[slot];
+  if (s->lead != (uint32_t)row) return;  // another record leads this slot
+  const uint32_t pending = s->pend;
+  SlotImage* img = &s_img[warp];
+  if (lane == 0) { img->count = s->count; img->n_items = s->n_items; }
+  if (lane < KMAX) { img->ids[lane] = s->ids[lane]; img->probs[lane] = s->probs[lane]; }
+  __syncwarp();
+  const bool fresh_slot = img->count == 0;
+  merge_warp(img, p.rec_ids + row * p.K, p.rec_p + row * p.K, p.K, lane);
+  uint32_t applied = 1;
+  for (long long i0 = (row + 1) & ~31ll; applied < pending && i0 < p.n_rows; i0 += 32) {
+    const long long i = i0 + lane;
+    const bool hit = i > row && i < p.n_rows && seg[i] == slot;
+    unsigned hits = __ballot_sync(FULL, hit);
+    while (hits) {
+      const int j = __ffs(hits) - 1;
+      hits &= hits - 1;
+      merge_warp(img, p.rec_ids + (i0 + j) * p.K, p.rec_p + (i0 + j) * p.K, p.K, lane);
+      ++applied;
+    }
+  }
+  const int n_items = (int)img->n_items;
+  if (lane < KMAX) {
+    s->ids[lane] = lane < n_items ? img->ids[lane] : 0;
+    s->probs[lane] = lane < n_items ? img->probs[lane] : 0.0f;
+  }
+  if (lane == 0) {
+    s->count = img->count;
+    s->n_items = img->n_items;
+    s->lead = NO_REC;
+    s->pend = 0;
+    atomicAdd(&p.stats[ST_RECORDS], (unsigned long long)applied);
+    if (fresh_slot) atomicAdd(&p.stats[ST_INSERTS], 1ull);
+  }
 }
 
 // ---------------------------------------------------------------------------
@@ -224,15 +369,19 @@ __global__ void table_dump_kernel(const Slot* table, unsigned long long n_slots,
   }
 }
 
-__global__ void table_load_kernel(Slot* table, unsigned long long mask, int max_probe, int K, const int* keys,
-                                  const uint32_t* counts, const int* n_items, const int* ids, const float* probs,
-                                  unsigned long long M, unsigned long long* stats) {
-  const unsigned long long i = (unsigned long long)blockIdx.x * blockDim.x + threadIdx.x;
-  if (i >= M) return;
-  int key[4];
-  for (int t = 0; t < 4; ++t) key[t] = keys[i * 4 + t];
-  const uint32_t slot = find_or_insert(table, mask, max_probe, key, stats);
-  if (slot == NO_SLOT) return;
+// One group of 8 lanes per entry.
+__global__ void __launch_bounds__(256) table_load_kernel(Slot* table, unsigned long long mask, int max_probe, int K,
+                                                         const int* keys, const uint32_t* counts, const int* n_items,
+                                                         const int* ids, const float* probs, unsigned long long M,
+                                                         unsigned long long* stats) {
+  const unsigned long long i = ((unsigned long long)blockIdx.x * blockDim.x + threadIdx.x) / GROUP;
+  const int gl = threadIdx.x & (GROUP - 1);
+  const bool live = i < M;
+  int key[4] = {-1, -1, -1, -1};
+  if (live)
+    for (int t = 0; t < 4; ++t) key[t] = keys[i * 4 + t];
+  const uint32_t slot = find_or_insert_group(table, mask, max_probe, key, live, stats);
+  if (!live || slot == NO_SLOT || gl != 0) return;
   Slot* s = &table[slot];
   s->count = counts[i];
   const int n = n_items[i] < K ? n_items[i] : K;
