@@ -52,6 +52,7 @@ extern "C" {
 #define STAND_E_WORKSPACE (-2) /* workspace missing, misaligned or too small */
 #define STAND_E_CUDA (-3)      /* a CUDA runtime call failed */
 #define STAND_E_STATE (-4)     /* call not valid in the current state */
+#define STAND_E_TOO_LARGE (-5) /* problem does not fit the library's built-in scratch buffer */
 
 typedef struct stand_ctx stand_ctx;
 
@@ -155,6 +156,36 @@ size_t stand_row_stats_scratch_bytes(int64_t rows, int32_t V, int32_t dtype, int
 int stand_row_stats(const void* dev_logits, int64_t rows, int32_t V, int32_t dtype, float temperature, int32_t topk,
                     void* dev_scratch, size_t scratch_bytes, float* dev_lse, int32_t* dev_ids, float* dev_values,
                     float* dev_probs, void* cu_stream);
+
+/* stand_row_stats for callers that cannot allocate device memory.  (The paper has no
+ * counterpart: this entry point exists for the library's users, not for the method.)
+ *
+ * Who needs it: code that runs where cudaMalloc is off limits -- inside a region
+ * that must not synchronise the device or grow its memory footprint (a serving loop
+ * with a fixed memory budget, a plugin that is handed buffers by its host and has no
+ * allocator of its own, a latency-critical path where an allocation could stall on
+ * other streams).  Such a caller still owns the input and the four outputs; only the
+ * scratch memory that stand_row_stats asks for is replaced by a buffer that is part
+ * of the library image: STAND_STATIC_SCRATCH_BYTES of device memory, held by every
+ * GPU that loads the library from load until the process exits.
+ *
+ * Same arguments, results and layouts as stand_row_stats, minus the scratch pair.
+ * Differences:
+ *   - Shapes whose scratch need (stand_row_stats_scratch_bytes) exceeds
+ *     STAND_STATIC_SCRATCH_BYTES are refused with STAND_E_TOO_LARGE; nothing is
+ *     launched.
+ *   - The first call on a device looks up the buffer's device address (once per
+ *     device, for the device that is current at the call) and caches it.  Make that
+ *     first call outside any stream capture.
+ *   - All calls on a device share the one buffer, and it keeps the previous call's
+ *     contents.  The kernels overwrite every scratch entry they later read, so no
+ *     clearing is needed; but two calls whose kernels overlap on the GPU (different
+ *     streams without an ordering between them) race on it.  Order such calls.
+ *   - No cudaMalloc, cudaFree or other allocating routine is called, here or below. */
+#define STAND_STATIC_SCRATCH_BYTES (8u << 20)
+int stand_row_stats_static(const void* dev_logits, int64_t rows, int32_t V, int32_t dtype, float temperature,
+                           int32_t topk, float* dev_lse, int32_t* dev_ids, float* dev_values, float* dev_probs,
+                           void* cu_stream);
 
 /* Synchronises the stream the context last used and copies the counters. */
 int stand_get_stats(stand_ctx* ctx, stand_stats* host_out);

@@ -18,9 +18,9 @@ DTYPE_F32, DTYPE_BF16 = 0, 1
 EXPORTS = [
     "stand_workspace_bytes", "stand_init", "stand_destroy", "stand_reset_sequences", "stand_verify_tree",
     "stand_ngram_update", "stand_ngram_update_bulk", "stand_draft_tree", "stand_step", "stand_step_host",
-    "stand_row_stats_scratch_bytes", "stand_row_stats", "stand_get_stats", "stand_last_path", "stand_tree_depth",
-    "stand_table_dump", "stand_table_load", "stand_state_dump", "stand_state_load", "stand_profile_row_pass",
-    "stand_launch_count", "stand_strerror",
+    "stand_row_stats_scratch_bytes", "stand_row_stats", "stand_row_stats_static", "stand_get_stats",
+    "stand_last_path", "stand_tree_depth", "stand_table_dump", "stand_table_load", "stand_state_dump",
+    "stand_state_load", "stand_profile_row_pass", "stand_launch_count", "stand_strerror",
 ]
 
 
@@ -72,6 +72,8 @@ def lib():
     L.stand_row_stats_scratch_bytes.restype = C.c_size_t
     L.stand_row_stats_scratch_bytes.argtypes = [i64, i32, i32, i32]
     L.stand_row_stats.argtypes = [vp, i64, i32, i32, f32, i32, vp, C.c_size_t, vp, vp, vp, vp, vp]
+    L.stand_row_stats_static.argtypes = [vp, i64, i32, i32, f32, i32, vp, vp, vp, vp, vp]
+    L.stand_row_stats_static.restype = C.c_int
     L.stand_get_stats.argtypes = [vp, C.POINTER(StandStats)]
     L.stand_last_path.argtypes = [vp, vp, vp, vp, vp]
     L.stand_tree_depth.argtypes = [vp]
@@ -328,3 +330,30 @@ def row_stats(logits, temperature, topk, stream=None):
                                  _ptr(probs), _stream(stream)), "stand_row_stats")
     (torch.cuda.current_stream() if stream is None else stream).synchronize()
     return lse, ids, vals, probs
+
+
+STATIC_SCRATCH_BYTES = 8 << 20
+
+
+def row_stats_static(logits, temperature, topk, out=None, stream=None):
+    """stand_row_stats_static: the row pass with the library's built-in scratch buffer, for callers that
+    cannot allocate device memory.  `out` = (lse, ids, values, probs) tensors the caller already owns;
+    when it is None they are made here (a convenience for tests -- the C call itself allocates nothing).
+    Raises StandError when the shape needs more scratch than the built-in buffer holds."""
+    import torch
+    assert logits.is_cuda and logits.is_contiguous() and logits.dim() == 2
+    assert logits.dtype in (torch.bfloat16, torch.float32)
+    rows, V = logits.shape
+    dtype = DTYPE_BF16 if logits.dtype == torch.bfloat16 else DTYPE_F32
+    dev = logits.device
+    if out is None:
+        out = (torch.empty(rows, dtype=torch.float32, device=dev),
+               torch.empty((rows, topk), dtype=torch.int32, device=dev),
+               torch.empty((rows, topk), dtype=torch.float32, device=dev),
+               torch.empty((rows, topk), dtype=torch.float32, device=dev))
+    lse, ids, vals, probs = out
+    with torch.cuda.device(dev):
+        _check(lib().stand_row_stats_static(_ptr(logits), rows, V, dtype, float(temperature), topk, _ptr(lse), _ptr(ids),
+                                            _ptr(vals), _ptr(probs), _stream(stream)), "stand_row_stats_static")
+    (torch.cuda.current_stream() if stream is None else stream).synchronize()
+    return out

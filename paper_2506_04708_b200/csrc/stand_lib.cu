@@ -3,6 +3,7 @@
 #include "../../include/stand.h"
 
 #include <cuda_runtime.h>
+#include <atomic>
 #include <new>
 #include <stdio.h>
 #include <string.h>
@@ -426,6 +427,31 @@ int stand_row_stats(const void* dev_logits, int64_t rows, int32_t V, int32_t dty
   return launch_ok();
 }
 
+// Scratch of stand_row_stats_static.  In host code this name is only a handle for
+// cudaGetSymbolAddress, never a device address.
+static __device__ __align__(256) unsigned char g_static_scratch[STAND_STATIC_SCRATCH_BYTES];
+constexpr int STATIC_MAX_DEVICES = 64;
+static std::atomic<void*> g_static_scratch_addr[STATIC_MAX_DEVICES];
+
+int stand_row_stats_static(const void* dev_logits, int64_t rows, int32_t V, int32_t dtype, float temperature,
+                           int32_t topk, float* dev_lse, int32_t* dev_ids, float* dev_values, float* dev_probs,
+                           void* cu_stream) {
+  const size_t need = stand_row_stats_scratch_bytes(rows, V, dtype, topk);
+  if (need == 0) return STAND_E_ARG;
+  if (need > (size_t)STAND_STATIC_SCRATCH_BYTES) return STAND_E_TOO_LARGE;
+  int dev = -1;
+  if (cudaGetDevice(&dev) != cudaSuccess) return STAND_E_CUDA;
+  if (dev < 0 || dev >= STATIC_MAX_DEVICES) return STAND_E_ARG;
+  void* scratch = g_static_scratch_addr[dev].load(std::memory_order_acquire);
+  if (!scratch) {
+    // first call on this device: resolve the buffer's address in this device's copy of the image
+    if (cudaGetSymbolAddress(&scratch, g_static_scratch) != cudaSuccess || !scratch) return STAND_E_CUDA;
+    g_static_scratch_addr[dev].store(scratch, std::memory_order_release);
+  }
+  return stand_row_stats(dev_logits, rows, V, dtype, temperature, topk, scratch, (size_t)STAND_STATIC_SCRATCH_BYTES, dev_lse,
+                         dev_ids, dev_values, dev_probs, cu_stream);
+}
+
 int stand_get_stats(stand_ctx* x, stand_stats* host_out) {
   if (!x || !host_out) return STAND_E_ARG;
   int rc = cuda_ok(cudaStreamSynchronize(x->last_stream));
@@ -558,6 +584,7 @@ const char* stand_strerror(int code) {
     case STAND_E_WORKSPACE: return "workspace missing, misaligned or too small";
     case STAND_E_CUDA: return "a CUDA runtime call failed";
     case STAND_E_STATE: return "call not valid in the current state";
+    case STAND_E_TOO_LARGE: return "problem does not fit the built-in scratch buffer";
     default: return "unknown error code";
   }
 }
