@@ -68,7 +68,7 @@ typedef struct {
   uint64_t seed;
   uint64_t table_slots;   /* power of two, >= 2; one slot = 128 bytes */
   const int32_t* parent;  /* HOST, [N]; parent[0] = -1; read during stand_init only */
-  int32_t chunks_per_unit; /* 0 = automatic; how many 1024-element chunks one warp streams */
+  int32_t reserved;        /* must be 0 */
   int32_t host_staging;    /* != 0: reserve a logits staging buffer for stand_step_host */
 } stand_config;
 
@@ -82,6 +82,7 @@ typedef struct {
   uint64_t lookups;         /* drafting lookups (one per tree node with children) */
   uint64_t lookup_hits[STAND_MAX_ORDER]; /* hits by order-1 */
   uint64_t max_probe_seen;  /* longest probe sequence */
+  uint64_t wait_timeouts;   /* non-zero: a bounded wait inside a kernel ran out (results of that step are invalid) */
 } stand_stats;
 
 /* Bytes of device workspace a configuration needs; 0 if the configuration is invalid. */
@@ -151,7 +152,9 @@ int stand_step_host(stand_ctx* ctx, const void* host_logits, int32_t* host_emitt
  * x/T (dev_lse [rows] float), and the top-k entries by (value descending, id
  * ascending): dev_ids [rows, topk] int32, dev_values [rows, topk] float (input
  * values), dev_probs [rows, topk] float (softmax probabilities).  dev_scratch must
- * hold stand_row_stats_scratch_bytes bytes, 256-byte aligned. */
+ * hold stand_row_stats_scratch_bytes bytes, 256-byte aligned.  Inputs are finite or
+ * -inf.  If a bounded wait inside the kernel runs out (never seen; it guards against a
+ * hang), every dev_lse entry is NaN and every id -1. */
 size_t stand_row_stats_scratch_bytes(int64_t rows, int32_t V, int32_t dtype, int32_t topk);
 int stand_row_stats(const void* dev_logits, int64_t rows, int32_t V, int32_t dtype, float temperature, int32_t topk,
                     void* dev_scratch, size_t scratch_bytes, float* dev_lse, int32_t* dev_ids, float* dev_values,
@@ -178,8 +181,8 @@ int stand_row_stats(const void* dev_logits, int64_t rows, int32_t V, int32_t dty
  *     device, for the device that is current at the call) and caches it.  Make that
  *     first call outside any stream capture.
  *   - All calls on a device share the one buffer, and it keeps the previous call's
- *     contents.  The kernels overwrite every scratch entry they later read, so no
- *     clearing is needed; but two calls whose kernels overlap on the GPU (different
+ *     contents.  Each call clears the one word that must start at zero and overwrites
+ *     every other scratch entry it later reads; but two calls whose kernels overlap on the GPU (different
  *     streams without an ordering between them) race on it.  Order such calls.
  *   - No cudaMalloc, cudaFree or other allocating routine is called, here or below. */
 #define STAND_STATIC_SCRATCH_BYTES (8u << 20)

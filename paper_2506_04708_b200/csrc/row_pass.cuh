@@ -1,33 +1,47 @@
-// Row pass: the one pass over the logits.  Temperature softmax statistics
-// (paper Sec. 5: sampling at temperature T) and the per-row top-k that the
-// N-gram module stores (Sec. 4.1), fused.
+// Row pass: the one pass over the logits (paper Sec. 5: sampling at temperature
+// T, i.e. softmax of x / T).
 //
-// Work unit = one warp streaming `cpu` consecutive 1024-entry chunks of one row.
-// Per chunk the warp writes (sum_v 2^(x_v*c - o), o) with c = log2(e)/T and o an
-// offset near the running maximum, so that a row's normaliser is rebuilt later
-// as sum_c s_c * 2^(o_c - o*) and prefix sums over chunks serve the inverse-CDF
-// sample.  Per unit the warp writes its k best (value, id) pairs; the per-row
-// top-k is the merge of the unit lists.  HBM-bound: every logit is read exactly once
-// with 16-byte loads that bypass L1; the next chunk is in flight while the
-// current one is reduced.
+// Per 1024-entry chunk of a row the pass writes (s, m): m = the chunk's largest
+// input value and s = sum_v 2^(x_v * c - o) with c = log2(e) / T and the integer
+// offset o = ceil(m * c).  A row's normaliser is rebuilt later as
+// sum_chunks s * 2^(o - o*), exactly (integer exponents); prefix sums over chunks
+// serve the inverse-CDF sample; and the chunk maxima bound the per-row top-k
+// (Sec. 4.1) so tightly that it can be finished afterwards from about k chunks, for
+// the few rows that need it (row_topk_warp below).
+//
+// The kernel is bound by HBM bandwidth: persistent CTAs (two per SM) walk a
+// contiguous range of 8-chunk tiles; one elected lane streams tiles into a ring of
+// shared-memory stages with bulk asynchronous copies (TMA) that complete on
+// mbarriers, marked evict-first in L2; eight consumer warps take one chunk of a
+// tile each.  The inner loop has no branches: packed bf16 max, packed fp32 FMA/ADD,
+// one ex2 per entry.
 #pragma once
 #include "common.cuh"
 
 namespace stand {
 
-constexpr int K1_THREADS = 256;
-constexpr int K1_WARPS = K1_THREADS / 32;
+constexpr int K1_CONSUMER_WARPS = 8;                       // = chunks per tile
+constexpr int K1_THREADS = (K1_CONSUMER_WARPS + 1) * 32;   // + the producer warp
+constexpr int TILE_CHUNKS = K1_CONSUMER_WARPS;
+constexpr int TILE_ELEMS = TILE_CHUNKS * CHUNK;
+constexpr int K1_SMEM_DATA = 96 * 1024;                    // ring bytes per CTA (two CTAs per SM)
+constexpr unsigned SPIN_LIMIT = 1u << 22;                  // bounded waits: about a second, then the kernel gives up
+
 constexpr int COMPACT_AT = 64;              // candidate count that triggers a compaction
 constexpr int CAND_CAP = COMPACT_AT + 256;  // a warp adds at most 32 lanes x 8 entries between checks
+
+// status word values written by a kernel that gave up waiting
+constexpr int K1_ERR_FULL_WAIT = 1, K1_ERR_EMPTY_WAIT = 2;
 
 struct RowPassParams {
   const void* logits;
   long long rows;
-  int V, n_chunks, cpu, upr;  // chunks per unit, units per row
-  float c;                    // log2(e) / T
-  int topk;
-  float2* pairs;  // [rows, n_chunks]  (sum, offset)
-  uint2* part;    // [rows, upr, topk] (value bits, id); id 0xFFFFFFFF = unused
+  int V, n_chunks;
+  int tiles_per_row;
+  long long total_tiles;
+  float c;          // log2(e) / T
+  float2* pairs;    // [rows, n_chunks]  (sum, chunk max)
+  int* status;      // device word, set non-zero if a bounded wait ran out (may be null)
 };
 
 __device__ __forceinline__ float ex2_approx(float x) {
@@ -36,82 +50,325 @@ __device__ __forceinline__ float ex2_approx(float x) {
   return y;
 }
 
-__device__ __forceinline__ uint4 ld_stream16(const void* p) {
-  uint4 v;
-  asm volatile("ld.global.nc.L1::no_allocate.v4.u32 {%0,%1,%2,%3}, [%4];"
-               : "=r"(v.x), "=r"(v.y), "=r"(v.z), "=r"(v.w)
-               : "l"(p));
-  return v;
+// Offset of a chunk with maximum m: the integer o = ceil(m * c); 0 for an all -inf chunk.
+__device__ __forceinline__ float chunk_offset(float m, float c) {
+  return m == -INFINITY ? 0.0f : ceilf(__fmul_rn(m, c));
+}
+
+// ---- packed fp32 pairs (sm_100: two fp32 lanes per instruction) ----------------
+__device__ __forceinline__ unsigned long long pack2(float lo, float hi) {
+  unsigned long long r;
+  asm("mov.b64 %0, {%1, %2};" : "=l"(r) : "f"(lo), "f"(hi));
+  return r;
+}
+__device__ __forceinline__ void unpack2(unsigned long long v, float& lo, float& hi) {
+  asm("mov.b64 {%0, %1}, %2;" : "=f"(lo), "=f"(hi) : "l"(v));
+}
+__device__ __forceinline__ unsigned long long fma2(unsigned long long a, unsigned long long b, unsigned long long c) {
+  unsigned long long d;
+  asm("fma.rn.f32x2 %0, %1, %2, %3;" : "=l"(d) : "l"(a), "l"(b), "l"(c));
+  return d;
+}
+__device__ __forceinline__ unsigned long long add2(unsigned long long a, unsigned long long b) {
+  unsigned long long d;
+  asm("add.rn.f32x2 %0, %1, %2;" : "=l"(d) : "l"(a), "l"(b));
+  return d;
+}
+
+__device__ __forceinline__ uint32_t max_bf16x2(uint32_t a, uint32_t b) {
+  uint32_t r;
+  asm("max.bf16x2 %0, %1, %2;" : "=r"(r) : "r"(a), "r"(b));
+  return r;
+}
+
+// Warp maximum of a float through the integer reduction unit.
+__device__ __forceinline__ float warp_max_redux(float v) {
+  const uint32_t key = ordered_bits(__float_as_uint(v));
+  uint32_t m;
+  asm volatile("redux.sync.max.u32 %0, %1, 0xffffffff;" : "=r"(m) : "r"(key));
+  const uint32_t bits = (m & 0x80000000u) ? (m ^ 0x80000000u) : ~m;
+  return __uint_as_float(bits);
 }
 
 template <int DT> struct ElemTraits;
 template <> struct ElemTraits<0> {  // float
   static constexpr int VEC = 4, ESIZE = 4;
   static constexpr uint32_t NEG_INF_WORD = 0xFF800000u;
-  __device__ static __forceinline__ void unpack(const uint4& d, float (&f)[4]) {
-    f[0] = __uint_as_float(d.x); f[1] = __uint_as_float(d.y);
-    f[2] = __uint_as_float(d.z); f[3] = __uint_as_float(d.w);
-  }
   __device__ static __forceinline__ float vmax(const uint4& d) {
     return fmaxf(fmaxf(__uint_as_float(d.x), __uint_as_float(d.y)),
                  fmaxf(__uint_as_float(d.z), __uint_as_float(d.w)));
+  }
+  // sum2 += 2^(x * c - o) for the 4 entries of d
+  __device__ static __forceinline__ void accumulate(const uint4& d, unsigned long long c2, unsigned long long no2,
+                                                    unsigned long long& sum2) {
+    float a, b;
+    unpack2(fma2(pack2(__uint_as_float(d.x), __uint_as_float(d.y)), c2, no2), a, b);
+    sum2 = add2(sum2, pack2(ex2_approx(a), ex2_approx(b)));
+    unpack2(fma2(pack2(__uint_as_float(d.z), __uint_as_float(d.w)), c2, no2), a, b);
+    sum2 = add2(sum2, pack2(ex2_approx(a), ex2_approx(b)));
   }
 };
 template <> struct ElemTraits<1> {  // bfloat16, two per word, lower index in the low half
   static constexpr int VEC = 8, ESIZE = 2;
   static constexpr uint32_t NEG_INF_WORD = 0xFF80FF80u;
+  __device__ static __forceinline__ uint32_t vmax_packed(const uint4& d) {
+    return max_bf16x2(max_bf16x2(d.x, d.y), max_bf16x2(d.z, d.w));
+  }
+  __device__ static __forceinline__ float unpack_max(uint32_t m) {
+    return fmaxf(__uint_as_float(m << 16), __uint_as_float(m & 0xFFFF0000u));
+  }
+  __device__ static __forceinline__ float vmax(const uint4& d) { return unpack_max(vmax_packed(d)); }
+  __device__ static __forceinline__ void word(uint32_t w, unsigned long long c2, unsigned long long no2,
+                                              unsigned long long& sum2) {
+    float a, b;
+    unpack2(fma2(pack2(__uint_as_float(w << 16), __uint_as_float(w & 0xFFFF0000u)), c2, no2), a, b);
+    sum2 = add2(sum2, pack2(ex2_approx(a), ex2_approx(b)));
+  }
+  __device__ static __forceinline__ void accumulate(const uint4& d, unsigned long long c2, unsigned long long no2,
+                                                    unsigned long long& sum2) {
+    word(d.x, c2, no2, sum2); word(d.y, c2, no2, sum2); word(d.z, c2, no2, sum2); word(d.w, c2, no2, sum2);
+  }
   __device__ static __forceinline__ void unpack(const uint4& d, float (&f)[8]) {
     f[0] = __uint_as_float(d.x << 16); f[1] = __uint_as_float(d.x & 0xFFFF0000u);
     f[2] = __uint_as_float(d.y << 16); f[3] = __uint_as_float(d.y & 0xFFFF0000u);
     f[4] = __uint_as_float(d.z << 16); f[5] = __uint_as_float(d.z & 0xFFFF0000u);
     f[6] = __uint_as_float(d.w << 16); f[7] = __uint_as_float(d.w & 0xFFFF0000u);
   }
-  __device__ static __forceinline__ uint32_t max2(uint32_t a, uint32_t b) {
-    uint32_t r;
-    asm("max.bf16x2 %0, %1, %2;" : "=r"(r) : "r"(a), "r"(b));
-    return r;
-  }
-  __device__ static __forceinline__ float vmax(const uint4& d) {
-    const uint32_t m = max2(max2(d.x, d.y), max2(d.z, d.w));
-    return fmaxf(__uint_as_float(m << 16), __uint_as_float(m & 0xFFFF0000u));
-  }
 };
 
-// The NV 16-byte vectors of lane `lane` in chunk `chunk`: vector i covers entries
-// chunk*1024 + i*32*VEC + lane*VEC .. +VEC.  Entries past V read as -inf.
-template <int DT, bool ALIGNED>
-__device__ __forceinline__ void load_chunk(const char* row, int V, int chunk, int lane,
-                                           uint4 (&d)[CHUNK / (32 * ElemTraits<DT>::VEC)]) {
+// (sum, max) of one chunk held as NV 16-byte vectors per lane; all lanes get the result.
+template <int DT, int NV>
+__device__ __forceinline__ float2 reduce_chunk(const uint4 (&v)[NV], float c) {
+  using TR = ElemTraits<DT>;
+  float lane_max;
+  if (DT == 1) {
+    uint32_t m = ElemTraits<1>::vmax_packed(v[0]);
+#pragma unroll
+    for (int i = 1; i < NV; ++i) m = max_bf16x2(m, ElemTraits<1>::vmax_packed(v[i]));
+    lane_max = ElemTraits<1>::unpack_max(m);
+  } else {
+    lane_max = TR::vmax(v[0]);
+#pragma unroll
+    for (int i = 1; i < NV; ++i) lane_max = fmaxf(lane_max, TR::vmax(v[i]));
+  }
+  const float cm = warp_max_redux(lane_max);
+  const float off = chunk_offset(cm, c);
+  const unsigned long long c2 = pack2(c, c), no2 = pack2(-off, -off);
+  unsigned long long sum2 = pack2(0.0f, 0.0f);
+#pragma unroll
+  for (int i = 0; i < NV; ++i) TR::accumulate(v[i], c2, no2, sum2);
+  float a, b;
+  unpack2(sum2, a, b);
+  return make_float2(warp_sum_f(a + b), cm);
+}
+
+// ---- mbarrier / bulk-copy primitives ---------------------------------------------
+__device__ __forceinline__ uint32_t smem_addr(const void* p) { return (uint32_t)__cvta_generic_to_shared(p); }
+__device__ __forceinline__ void mbar_init(uint32_t bar, uint32_t count) {
+  asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(bar), "r"(count) : "memory");
+}
+__device__ __forceinline__ void mbar_arrive(uint32_t bar) {
+  asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(bar) : "memory");
+}
+__device__ __forceinline__ void mbar_expect_tx(uint32_t bar, uint32_t bytes) {
+  asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(bar), "r"(bytes) : "memory");
+}
+__device__ __forceinline__ bool mbar_try_wait(uint32_t bar, uint32_t parity) {
+  uint32_t ok;
+  asm volatile(
+      "{\n\t.reg .pred p;\n\t"
+      "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
+      "selp.u32 %0, 1, 0, p;\n\t}"
+      : "=r"(ok)
+      : "r"(bar), "r"(parity)
+      : "memory");
+  return ok != 0;
+}
+// Bounded wait; false if the limit ran out or another thread of the CTA already gave up.
+__device__ __forceinline__ bool mbar_wait_bounded(uint32_t bar, uint32_t parity, const volatile int* abort_flag) {
+  for (unsigned spin = 0; spin < SPIN_LIMIT; ++spin) {
+    if (mbar_try_wait(bar, parity)) return true;
+    if (*abort_flag) return false;
+  }
+  return false;
+}
+__device__ __forceinline__ unsigned long long l2_evict_first_policy() {
+  unsigned long long pol;
+  asm volatile("createpolicy.fractional.L2::evict_first.b64 %0, 1.0;" : "=l"(pol));
+  return pol;
+}
+// global -> shared bulk copy (16-byte aligned addresses, size a multiple of 16), completes on `bar`
+__device__ __forceinline__ void bulk_load(uint32_t dst, const void* src, uint32_t bytes, uint32_t bar,
+                                          unsigned long long policy) {
+  asm volatile(
+      "cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes.L2::cache_hint [%0], [%1], %2, [%3], %4;"
+      ::"r"(dst), "l"(src), "r"(bytes), "r"(bar), "l"(policy)
+      : "memory");
+}
+
+// ---------------------------------------------------------------------------------
+// The streaming kernel.  Requires a 16-byte aligned base and V * sizeof(elem) a
+// multiple of 16 (the host checks and falls back to row_pass_plain_kernel).
+// ---------------------------------------------------------------------------------
+template <int DT>
+__global__ void __launch_bounds__(K1_THREADS, 2) row_pass_kernel(const RowPassParams p) {
   using TR = ElemTraits<DT>;
   constexpr int VEC = TR::VEC, NV = CHUNK / (32 * VEC);
-#pragma unroll
-  for (int i = 0; i < NV; ++i) {
-    const int idx = chunk * CHUNK + i * 32 * VEC + lane * VEC;
-    if (ALIGNED) {
-      if (idx < V) d[i] = ld_stream16(row + (size_t)idx * TR::ESIZE);
-      else d[i] = make_uint4(TR::NEG_INF_WORD, TR::NEG_INF_WORD, TR::NEG_INF_WORD, TR::NEG_INF_WORD);
-    } else {
-      uint32_t w[4];
-      if (DT == 0) {
-#pragma unroll
-        for (int e = 0; e < 4; ++e)
-          w[e] = idx + e < V ? __ldg((const uint32_t*)row + idx + e) : 0xFF800000u;
-      } else {
-#pragma unroll
-        for (int e = 0; e < 4; ++e) {
-          const uint32_t lo = idx + 2 * e < V ? __ldg((const unsigned short*)row + idx + 2 * e) : 0xFF80u;
-          const uint32_t hi = idx + 2 * e + 1 < V ? __ldg((const unsigned short*)row + idx + 2 * e + 1) : 0xFF80u;
-          w[e] = lo | (hi << 16);
+  constexpr int STAGE_BYTES = TILE_ELEMS * TR::ESIZE;
+  constexpr int STAGES = K1_SMEM_DATA / STAGE_BYTES;
+  static_assert(STAGES >= 2, "ring too small");
+  extern __shared__ __align__(128) unsigned char smem[];
+  __shared__ __align__(8) unsigned long long s_full[STAGES], s_empty[STAGES];
+  __shared__ volatile int s_abort;
+
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  const long long t0 = (long long)blockIdx.x * p.total_tiles / gridDim.x;
+  const long long t1 = (long long)(blockIdx.x + 1) * p.total_tiles / gridDim.x;
+  const long long n_tiles = t1 - t0;
+  if (threadIdx.x == 0) {
+    s_abort = 0;
+    for (int s = 0; s < STAGES; ++s) {
+      mbar_init(smem_addr(&s_full[s]), 1);
+      mbar_init(smem_addr(&s_empty[s]), K1_CONSUMER_WARPS);
+    }
+    asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+  }
+  __syncthreads();
+  const size_t row_bytes = (size_t)p.V * TR::ESIZE;
+
+  if (warp == K1_CONSUMER_WARPS) {
+    // ---- producer: one lane keeps the ring full ------------------------------------
+    if (lane == 0) {
+      const unsigned long long policy = l2_evict_first_policy();
+      long long issued = 0;
+      for (long long i = 0; i < n_tiles; ++i) {
+        const int s = (int)(i % STAGES);
+        const uint32_t round = (uint32_t)(i / STAGES);
+        if (!mbar_wait_bounded(smem_addr(&s_empty[s]), (round & 1u) ^ 1u, &s_abort)) {
+          if (!s_abort && p.status) atomicExch(p.status, K1_ERR_EMPTY_WAIT);
+          s_abort = 1;
+          break;
+        }
+        const long long g = t0 + i;
+        const long long row = g / p.tiles_per_row;
+        const int t = (int)(g - row * p.tiles_per_row);
+        const size_t at = (size_t)t * STAGE_BYTES;
+        const uint32_t bytes = (uint32_t)(row_bytes - at < (size_t)STAGE_BYTES ? row_bytes - at : (size_t)STAGE_BYTES);
+        const uint32_t bar = smem_addr(&s_full[s]);
+        mbar_expect_tx(bar, bytes);
+        bulk_load(smem_addr(smem + (size_t)s * STAGE_BYTES), (const char*)p.logits + (size_t)row * row_bytes + at, bytes, bar,
+                  policy);
+        issued = i + 1;
+      }
+      if (s_abort) {
+        // leave no copy in flight behind: wait (bounded) for the stages that were issued last
+        for (long long i = issued > STAGES ? issued - STAGES : 0; i < issued; ++i) {
+          const uint32_t bar = smem_addr(&s_full[(int)(i % STAGES)]);
+          for (unsigned spin = 0; spin < SPIN_LIMIT && !mbar_try_wait(bar, (uint32_t)(i / STAGES) & 1u); ++spin) {}
         }
       }
-      d[i] = make_uint4(w[0], w[1], w[2], w[3]);
+    }
+    return;
+  }
+
+  // ---- consumers: warp w takes chunk w of every tile -----------------------------------
+  const float c = p.c;
+  for (long long i = 0; i < n_tiles; ++i) {
+    const int s = (int)(i % STAGES);
+    const uint32_t round = (uint32_t)(i / STAGES);
+    const bool landed = mbar_wait_bounded(smem_addr(&s_full[s]), round & 1u, &s_abort);
+    if (!__all_sync(FULL, landed)) {  // warp-uniform: the lanes leave together
+      if (lane == 0) {
+        if (!s_abort && p.status) atomicExch(p.status, K1_ERR_FULL_WAIT);
+        s_abort = 1;
+      }
+      break;
+    }
+    const long long g = t0 + i;
+    const long long row = g / p.tiles_per_row;
+    const int t = (int)(g - row * p.tiles_per_row);
+    const int chunk = t * TILE_CHUNKS + warp;
+    if (chunk < p.n_chunks) {
+      const uint4* src = reinterpret_cast<const uint4*>(smem + (size_t)s * STAGE_BYTES + (size_t)warp * CHUNK * TR::ESIZE);
+      uint4 v[NV];
+#pragma unroll
+      for (int k = 0; k < NV; ++k) v[k] = src[k * 32 + lane];
+      if ((chunk + 1) * CHUNK > p.V) {  // the row's ragged last chunk: entries past V count as -inf
+#pragma unroll
+        for (int k = 0; k < NV; ++k)
+          if (chunk * CHUNK + (k * 32 + lane) * VEC >= p.V)
+            v[k] = make_uint4(TR::NEG_INF_WORD, TR::NEG_INF_WORD, TR::NEG_INF_WORD, TR::NEG_INF_WORD);
+      }
+      __syncwarp();
+      if (lane == 0) mbar_arrive(smem_addr(&s_empty[s]));  // the data is in registers: hand the stage back early
+      const float2 r = reduce_chunk<DT, NV>(v, c);
+      if (lane == 0) p.pairs[row * p.n_chunks + chunk] = r;
+    } else {
+      if (lane == 0) mbar_arrive(smem_addr(&s_empty[s]));
     }
   }
 }
 
+// Fallback for rows that are not 16-byte aligned: one warp per (row, chunk), scalar loads.
+template <int DT>
+__global__ void __launch_bounds__(256) row_pass_plain_kernel(const RowPassParams p) {
+  const int lane = threadIdx.x & 31;
+  const long long unit = (long long)blockIdx.x * 8 + (threadIdx.x >> 5);
+  if (unit >= p.rows * p.n_chunks) return;
+  const long long row = unit / p.n_chunks;
+  const int chunk = (int)(unit - row * p.n_chunks);
+  float x[CHUNK / 32];
+  float lane_max = -INFINITY;
+#pragma unroll
+  for (int j = 0; j < CHUNK / 32; ++j) {
+    const int v = chunk * CHUNK + j * 32 + lane;
+    x[j] = v < p.V ? load_logit(p.logits, DT, row * (long long)p.V + v) : -INFINITY;
+    lane_max = fmaxf(lane_max, x[j]);
+  }
+  const float cm = warp_max_redux(lane_max);
+  const float off = chunk_offset(cm, p.c);
+  float sum = 0.0f;
+#pragma unroll
+  for (int j = 0; j < CHUNK / 32; ++j) sum += ex2_approx(fmaf(x[j], p.c, -off));
+  sum = warp_sum_f(sum);
+  if (lane == 0) p.pairs[unit] = make_float2(sum, cm);
+}
+
+// ---------------------------------------------------------------------------
+// Per-row results from the chunk pairs.
+// ---------------------------------------------------------------------------
+struct RowNorm {
+  float off;  // o* = largest chunk offset (an integer)
+  double Z;   // sum_c s_c 2^(o_c - o*)
+};
+
+// All lanes of a warp call this; every lane gets the result.
+__device__ __forceinline__ RowNorm row_normaliser(const float2* pairs, int n_chunks, float c, int lane) {
+  float om = -INFINITY;
+  for (int ch = lane; ch < n_chunks; ch += 32) {
+    const float2 pr = pairs[ch];
+    if (pr.x > 0.0f) om = fmaxf(om, chunk_offset(pr.y, c));
+  }
+  om = warp_max_f(om);
+  double z = 0.0;
+  for (int ch = lane; ch < n_chunks; ch += 32) {
+    const float2 pr = pairs[ch];
+    if (pr.x > 0.0f) z += scalbn((double)pr.x, (int)(chunk_offset(pr.y, c) - om));
+  }
+  RowNorm r;
+  r.off = om;
+  r.Z = warp_sum_d(z);
+  return r;
+}
+
+// Mass of one chunk relative to the row offset `off` (before division by Z).
+__device__ __forceinline__ double chunk_mass(float2 pr, float c, float off) {
+  return pr.x > 0.0f ? scalbn((double)pr.x, (int)(chunk_offset(pr.y, c) - off)) : 0.0;
+}
+
 // Keeps the k best of the n buffered candidates at buf[0..k), best first; returns
-// the new threshold (the k-th value, or -inf while fewer than k are known).
-__device__ __forceinline__ float compact_topk(uint2* buf, int* cnt, int n, int k, int lane) {
+// the new threshold (the k-th value, or `floor` while fewer than k are known).
+__device__ __forceinline__ float compact_topk(uint2* buf, int* cnt, int n, int k, int lane, float floor) {
   const int keep = n < k ? n : k;
   for (int r = 0; r < keep; ++r) {
     unsigned long long best = 0ull;
@@ -131,141 +388,9 @@ __device__ __forceinline__ float compact_topk(uint2* buf, int* cnt, int n, int k
   }
   if (lane == 0) *cnt = keep;
   __syncwarp();
-  return keep == k ? __uint_as_float(buf[k - 1].x) : -INFINITY;
+  return keep == k ? fmaxf(floor, __uint_as_float(buf[k - 1].x)) : floor;
 }
 
-template <int DT, bool ALIGNED>
-__global__ void __launch_bounds__(K1_THREADS) row_pass_kernel(const RowPassParams p) {
-  using TR = ElemTraits<DT>;
-  constexpr int VEC = TR::VEC, NV = CHUNK / (32 * VEC);
-  __shared__ uint2 s_buf[K1_WARPS][CAND_CAP];
-  __shared__ int s_cnt[K1_WARPS];
-
-  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-  const long long unit = (long long)blockIdx.x * K1_WARPS + warp;
-  if (unit >= p.rows * p.upr) return;  // warps are independent: no block-wide barrier below
-  const long long row = unit / p.upr;
-  const int split = (int)(unit - row * p.upr);
-  const int c0 = split * p.cpu;
-  const int c1 = min(c0 + p.cpu, p.n_chunks);
-  const char* rowp = (const char*)p.logits + (size_t)row * (size_t)p.V * TR::ESIZE;
-  uint2* buf = s_buf[warp];
-  int* cnt = &s_cnt[warp];
-  if (lane == 0) *cnt = 0;
-  __syncwarp();
-
-  const float c = p.c;
-  const float span = 64.0f / c;  // re-centre when an entry exceeds the offset by 2^64
-  float tau = -INFINITY;         // candidates must reach this value
-  float off = 0.0f;              // current offset o (log2 domain)
-  float guard = -INFINITY;       // entries above this value force a new offset
-  bool first = true;
-
-  uint4 cur[NV], nxt[NV];
-  load_chunk<DT, ALIGNED>(rowp, p.V, c0, lane, cur);
-  for (int ch = c0; ch < c1; ++ch) {
-    if (ch + 1 < c1) load_chunk<DT, ALIGNED>(rowp, p.V, ch + 1, lane, nxt);
-
-    float sum = 0.0f;
-    bool over = first;
-    float lane_max = -INFINITY;
-#pragma unroll
-    for (int i = 0; i < NV; ++i) {
-      float f[VEC];
-      TR::unpack(cur[i], f);
-      const float vm = TR::vmax(cur[i]);
-      lane_max = fmaxf(lane_max, vm);
-      const bool hit = vm >= tau;
-      over |= vm > guard;
-      if (__any_sync(FULL, hit)) {  // rare after the first vectors of a unit
-        if (hit) {
-          const int idx0 = ch * CHUNK + i * 32 * VEC + lane * VEC;
-#pragma unroll
-          for (int e = 0; e < VEC; ++e) {
-            if (f[e] >= tau && idx0 + e < p.V) {
-              const int pos = atomicAdd(cnt, 1);
-              const float canon = f[e] == 0.0f ? 0.0f : f[e];  // -0 and +0 are one value
-              buf[pos] = make_uint2(__float_as_uint(canon), (uint32_t)(idx0 + e));
-            }
-          }
-        }
-        __syncwarp();
-        const int n = *(volatile int*)cnt;
-        if (n >= COMPACT_AT) tau = compact_topk(buf, cnt, n, p.topk, lane);
-      }
-#pragma unroll
-      for (int e = 0; e < VEC; ++e) sum += ex2_approx(fmaf(f[e], c, -off));
-    }
-    if (__any_sync(FULL, over)) {
-      // new offset from this chunk's maximum; redo the chunk's sum with it
-      const float cm = warp_max_f(lane_max);
-      off = cm == -INFINITY ? 0.0f : cm * c;
-      guard = cm == -INFINITY ? -INFINITY : cm + span;
-      first = false;
-      sum = 0.0f;
-#pragma unroll
-      for (int i = 0; i < NV; ++i) {
-        float f[VEC];
-        TR::unpack(cur[i], f);
-#pragma unroll
-        for (int e = 0; e < VEC; ++e) sum += ex2_approx(fmaf(f[e], c, -off));
-      }
-    }
-    sum = warp_sum_f(sum);
-    if (lane == 0) p.pairs[row * p.n_chunks + ch] = make_float2(sum, off);
-#pragma unroll
-    for (int i = 0; i < NV; ++i) cur[i] = nxt[i];
-  }
-
-  const int n = *(volatile int*)cnt;
-  const int keep = n < p.topk ? n : p.topk;
-  if (n > 0) compact_topk(buf, cnt, n, p.topk, lane);
-  if (lane < p.topk) {
-    p.part[(row * p.upr + split) * p.topk + lane] = lane < keep ? buf[lane] : make_uint2(0u, 0xFFFFFFFFu);
-  }
-}
-
-// ---------------------------------------------------------------------------
-// Per-row results from the unit partials (used by the context-free row-stats
-// entry point; the verification kernel does the same for the rows it needs).
-// ---------------------------------------------------------------------------
-struct RowNorm {
-  float off;  // o* = largest chunk offset
-  double Z;   // sum_c s_c 2^(o_c - o*)
-};
-
-// All lanes of a warp call this; every lane gets the result.
-__device__ __forceinline__ RowNorm row_normaliser(const float2* pairs, int n_chunks, int lane) {
-  float om = -INFINITY;
-  for (int c = lane; c < n_chunks; c += 32) {
-    const float2 pr = pairs[c];
-    if (pr.x > 0.0f) om = fmaxf(om, pr.y);
-  }
-  om = warp_max_f(om);
-  double z = 0.0;
-  for (int c = lane; c < n_chunks; c += 32) {
-    const float2 pr = pairs[c];
-    if (pr.x > 0.0f) z += (double)pr.x * exp2((double)pr.y - (double)om);
-  }
-  RowNorm r;
-  r.off = om;
-  r.Z = warp_sum_d(z);
-  return r;
-}
-
-// k-th round of a merge of unit lists without marking: the largest key strictly
-// below `below`.  All lanes call; every lane gets (key, value bits, id).
-__device__ __forceinline__ unsigned long long next_best(const uint2* part, int n_entries, unsigned long long below,
-                                                       int lane) {
-  unsigned long long best = 0ull;
-  for (int i = lane; i < n_entries; i += 32) {
-    const uint2 e = part[i];
-    if (e.y == 0xFFFFFFFFu) continue;
-    const unsigned long long key = select_key(e.x, e.y);
-    if (key < below && key > best) best = key;
-  }
-  return warp_max_u64(best);
-}
 // inverse of select_key
 __device__ __forceinline__ uint32_t key_id(unsigned long long key) { return ~(uint32_t)key; }
 __device__ __forceinline__ float key_value(unsigned long long key) {
@@ -274,11 +399,95 @@ __device__ __forceinline__ float key_value(unsigned long long key) {
   return __uint_as_float(bits);
 }
 
+// Sec. 4.1: the k entries of one row that the table keeps, by (value descending, id
+// ascending), exact.  The k-th largest chunk maximum is a lower bound of the k-th
+// largest entry (k different chunks hold an entry at least that large), so only
+// chunks whose maximum reaches it can hold a top-k entry: about k of them are read
+// again.  Called by all lanes of a warp; buf/cnt are the warp's own shared memory
+// (CAND_CAP entries).  On return buf[0..n) holds the entries, best first; returns n.
+__device__ __forceinline__ int row_topk_warp(const void* logits, int dtype, long long row, int V, const float2* pairs,
+                                             int n_chunks, int k, uint2* buf, int* cnt, int lane) {
+  // the k-th largest chunk maximum (chunk index breaks ties, so keys are distinct)
+  float tau = -INFINITY;
+  if (n_chunks >= k) {
+    unsigned long long below = ~0ull;
+    for (int r = 0; r < k; ++r) {
+      unsigned long long best = 0ull;
+      for (int ch = lane; ch < n_chunks; ch += 32) {
+        const unsigned long long key = select_key(__float_as_uint(pairs[ch].y), (uint32_t)ch);
+        if (key < below && key > best) best = key;
+      }
+      below = warp_max_u64(best);
+    }
+    tau = key_value(below);
+  }
+  const float floor = tau;
+  if (lane == 0) *cnt = 0;
+  __syncwarp();
+  const bool wide = dtype == 1 ? (((uintptr_t)logits & 15) == 0 && (V & 7) == 0)
+                               : (((uintptr_t)logits & 15) == 0 && (V & 3) == 0);
+  for (int c0 = 0; c0 < n_chunks; c0 += 32) {
+    const int mych = c0 + lane;
+    unsigned todo = __ballot_sync(FULL, mych < n_chunks && pairs[mych < n_chunks ? mych : 0].y >= floor);
+    while (todo) {
+      const int ch = c0 + __ffs(todo) - 1;
+      todo &= todo - 1;
+      // 1024 entries, 32 per lane, in 4 steps of 8 (at most 256 pushes between compaction checks)
+#pragma unroll 1
+      for (int step = 0; step < 4; ++step) {
+        float f[8];
+        int idx[8];
+        if (wide && dtype == 1) {
+          const int i0 = ch * CHUNK + step * 256 + lane * 8;
+          uint4 d = make_uint4(0xFF80FF80u, 0xFF80FF80u, 0xFF80FF80u, 0xFF80FF80u);
+          if (i0 < V) d = __ldg(reinterpret_cast<const uint4*>((const unsigned short*)logits + row * (long long)V + i0));
+          ElemTraits<1>::unpack(d, f);
+#pragma unroll
+          for (int e = 0; e < 8; ++e) idx[e] = i0 + e;
+        } else if (wide) {
+          const int i0 = ch * CHUNK + step * 256 + lane * 8;
+#pragma unroll
+          for (int h = 0; h < 2; ++h) {
+            uint4 d = make_uint4(0xFF800000u, 0xFF800000u, 0xFF800000u, 0xFF800000u);
+            if (i0 + 4 * h < V) d = __ldg(reinterpret_cast<const uint4*>((const float*)logits + row * (long long)V + i0 + 4 * h));
+            f[4 * h] = __uint_as_float(d.x); f[4 * h + 1] = __uint_as_float(d.y);
+            f[4 * h + 2] = __uint_as_float(d.z); f[4 * h + 3] = __uint_as_float(d.w);
+          }
+#pragma unroll
+          for (int e = 0; e < 8; ++e) idx[e] = i0 + e;
+        } else {
+#pragma unroll
+          for (int e = 0; e < 8; ++e) {
+            idx[e] = ch * CHUNK + step * 256 + e * 32 + lane;
+            f[e] = idx[e] < V ? load_logit(logits, dtype, row * (long long)V + idx[e]) : -INFINITY;
+          }
+        }
+#pragma unroll
+        for (int e = 0; e < 8; ++e) {
+          if (f[e] >= tau && idx[e] < V) {
+            const int pos = atomicAdd(cnt, 1);
+            const float canon = f[e] == 0.0f ? 0.0f : f[e];  // -0 and +0 are one value
+            buf[pos] = make_uint2(__float_as_uint(canon), (uint32_t)idx[e]);
+          }
+        }
+        __syncwarp();
+        const int n = *(volatile int*)cnt;
+        if (n >= COMPACT_AT) tau = compact_topk(buf, cnt, n, k, lane, floor);
+      }
+    }
+  }
+  const int n = *(volatile int*)cnt;
+  if (n > 0) compact_topk(buf, cnt, n, k, lane, floor);
+  return n < k ? n : k;
+}
+
 struct RowFinalizeParams {
+  const void* logits;
+  int dtype, V;
   const float2* pairs;
-  const uint2* part;
+  const int* status;  // non-zero: the row pass gave up on a wait, its pairs are not to be trusted
   long long rows;
-  int n_chunks, upr, topk;
+  int n_chunks, topk;
   float c;
   float* lse;
   int* ids;
@@ -286,29 +495,39 @@ struct RowFinalizeParams {
   float* probs;
 };
 
-__global__ void __launch_bounds__(256) row_finalize_kernel(const RowFinalizeParams p) {
-  const int lane = threadIdx.x & 31;
-  const long long row = (long long)blockIdx.x * 8 + (threadIdx.x >> 5);
+constexpr int FIN_WARPS = 4;
+__global__ void __launch_bounds__(FIN_WARPS * 32) row_finalize_kernel(const RowFinalizeParams p) {
+  __shared__ uint2 s_buf[FIN_WARPS][CAND_CAP];
+  __shared__ int s_cnt[FIN_WARPS];
+  const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+  const long long row = (long long)blockIdx.x * FIN_WARPS + warp;
   if (row >= p.rows) return;
-  const RowNorm nm = row_normaliser(p.pairs + row * p.n_chunks, p.n_chunks, lane);
-  if (lane == 0) p.lse[row] = (float)(((double)nm.off + log2(nm.Z)) * 0.6931471805599453);
-  const uint2* part = p.part + row * p.upr * p.topk;
-  unsigned long long below = ~0ull;
-  for (int r = 0; r < p.topk; ++r) {
-    const unsigned long long key = next_best(part, p.upr * p.topk, below, lane);
-    if (lane == 0) {
-      if (key == 0ull) {
-        p.ids[row * p.topk + r] = -1;
-        p.values[row * p.topk + r] = 0.0f;
-        p.probs[row * p.topk + r] = 0.0f;
-      } else {
-        const float x = key_value(key);
-        p.ids[row * p.topk + r] = (int)key_id(key);
-        p.values[row * p.topk + r] = x;
-        p.probs[row * p.topk + r] = (float)(exp2((double)x * (double)p.c - (double)nm.off) / nm.Z);
-      }
+  if (*p.status != 0) {  // report the failure in-band: NaN and no entries
+    if (lane == 0) p.lse[row] = __int_as_float(0x7FC00000);
+    if (lane < p.topk) {
+      p.ids[row * p.topk + lane] = -1;
+      p.values[row * p.topk + lane] = 0.0f;
+      p.probs[row * p.topk + lane] = 0.0f;
     }
-    if (key == 0ull) below = 0ull; else below = key;
+    return;
+  }
+  const float2* pairs = p.pairs + row * p.n_chunks;
+  const RowNorm nm = row_normaliser(pairs, p.n_chunks, p.c, lane);
+  if (lane == 0) p.lse[row] = (float)(((double)nm.off + log2(nm.Z)) * 0.6931471805599453);
+  const int n = row_topk_warp(p.logits, p.dtype, row, p.V, pairs, p.n_chunks, p.topk, s_buf[warp], &s_cnt[warp], lane);
+  if (lane < p.topk) {
+    const long long at = row * p.topk + lane;
+    if (lane < n) {
+      const uint2 e = s_buf[warp][lane];
+      const float x = __uint_as_float(e.x);
+      p.ids[at] = (int)e.y;
+      p.values[at] = x;
+      p.probs[at] = (float)(exp2((double)x * (double)p.c - (double)nm.off) / nm.Z);
+    } else {
+      p.ids[at] = -1;
+      p.values[at] = 0.0f;
+      p.probs[at] = 0.0f;
+    }
   }
 }
 

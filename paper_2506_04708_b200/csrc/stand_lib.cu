@@ -21,14 +21,14 @@ namespace {
 constexpr int BULK_ROWS = 16384;  // rows per batch of the bulk update
 
 struct Layout {
-  size_t table, topo, tail, len, tree, cand_n, cand_id, cand_phi, pairs, part, emitted, n_path, path, rec_ctx, rec_ids,
-      rec_p, rec_slot, stats, scratch64, staging, total;
+  size_t table, topo, tail, len, tree, cand_n, cand_id, cand_phi, pairs, emitted, n_path, path, rec_ctx, rec_ids,
+      rec_p, rec_slot, stats, status, staging, total;
 };
 
 inline size_t align_up(size_t x) { return (x + 255) & ~(size_t)255; }
 
 struct Derived {
-  int D, n_chunks, cpu, upr;
+  int D, n_chunks;
   int parent[NODES_MAX], first_child[NODES_MAX], n_children[NODES_MAX], depth[NODES_MAX], level_start[DEPTH_MAX + 2];
 };
 
@@ -37,7 +37,7 @@ bool derive(const stand_config* c, Derived* d) {
   if (c->B < 1 || c->N < 1 || c->N > STAND_MAX_NODES || c->V < 2 || c->V > STAND_MAX_VOCAB) return false;
   if (c->topk < 1 || c->topk > STAND_MAX_TOPK || c->order_max < 1 || c->order_max > STAND_MAX_ORDER) return false;
   if (c->dtype != STAND_DTYPE_F32 && c->dtype != STAND_DTYPE_BF16) return false;
-  if (!(c->temperature > 0.0f) || c->max_probe < 0 || c->chunks_per_unit < 0) return false;
+  if (!(c->temperature > 0.0f) || c->max_probe < 0 || c->reserved != 0) return false;
   if (c->table_slots < 2 || (c->table_slots & (c->table_slots - 1)) != 0 || c->table_slots > (1ull << 32) - 2) return false;
   if (!c->parent || c->parent[0] != -1) return false;
   if ((long long)c->B * c->N > (1ll << 31) / 4) return false;
@@ -62,16 +62,6 @@ bool derive(const stand_config* c, Derived* d) {
   for (int l = 0; l <= d->D + 1; ++l) d->level_start[l] = c->N;
   for (int u = c->N - 1; u >= 0; --u) d->level_start[d->depth[u]] = u;
   d->n_chunks = (c->V + CHUNK - 1) / CHUNK;
-  if (c->chunks_per_unit > 0) d->cpu = c->chunks_per_unit < d->n_chunks ? c->chunks_per_unit : d->n_chunks;
-  else {
-    // enough units to fill 148 SMs x 24 warps about twice over, units as long as that allows
-    const long long total = (long long)c->B * c->N * d->n_chunks;
-    long long cpu = (total + 7103) / 7104;
-    if (cpu < 1) cpu = 1;
-    if (cpu > d->n_chunks) cpu = d->n_chunks;
-    d->cpu = (int)cpu;
-  }
-  d->upr = (d->n_chunks + d->cpu - 1) / d->cpu;
   return true;
 }
 
@@ -92,7 +82,6 @@ void layout_of(const stand_config* c, const Derived* d, Layout* L) {
   L->cand_id = take(B * N * K * 4);
   L->cand_phi = take(B * N * K * 4);
   L->pairs = take(B * N * (size_t)d->n_chunks * sizeof(float2));
-  L->part = take(B * N * (size_t)d->upr * K * sizeof(uint2));
   L->emitted = take(B * W * 4);
   L->n_path = take(B * 4);
   L->path = take(B * W * 4);
@@ -101,7 +90,7 @@ void layout_of(const stand_config* c, const Derived* d, Layout* L) {
   L->rec_p = take(B * W * K * 4);
   L->rec_slot = take(rec_rows * n * 4);
   L->stats = take(ST_COUNT * 8);
-  L->scratch64 = take(64);
+  L->status = take(64);
   L->staging = take(c->host_staging ? B * N * (size_t)c->V * esize_of(c->dtype) : 0);
   L->total = at;
 }
@@ -141,21 +130,48 @@ bool rows_aligned(const void* base, int V, int dtype) {
   return ((uintptr_t)base % 16 == 0) && (((size_t)V * es) % 16 == 0);
 }
 
-int launch_row_pass(const void* logits, long long rows, int V, int dtype, int n_chunks, int cpu, int upr, float c, int topk,
-                    float2* pairs, uint2* part, cudaStream_t st) {
+// The streaming kernel needs more dynamic shared memory than the default limit: raise it once per device.
+constexpr int MAX_DEVICES = 64;
+std::atomic<int> g_k1_ready[MAX_DEVICES];
+std::atomic<int> g_sm_count[MAX_DEVICES];
+
+int prepare_device(int* sm_count) {
+  int dev = -1;
+  if (cudaGetDevice(&dev) != cudaSuccess) return STAND_E_CUDA;
+  if (dev < 0 || dev >= MAX_DEVICES) return STAND_E_ARG;
+  if (!g_k1_ready[dev].load(std::memory_order_acquire)) {
+    int sms = 0;
+    if (cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess || sms < 1) return STAND_E_CUDA;
+    if (cudaFuncSetAttribute(row_pass_kernel<0>, cudaFuncAttributeMaxDynamicSharedMemorySize, K1_SMEM_DATA) != cudaSuccess)
+      return STAND_E_CUDA;
+    if (cudaFuncSetAttribute(row_pass_kernel<1>, cudaFuncAttributeMaxDynamicSharedMemorySize, K1_SMEM_DATA) != cudaSuccess)
+      return STAND_E_CUDA;
+    g_sm_count[dev].store(sms, std::memory_order_relaxed);
+    g_k1_ready[dev].store(1, std::memory_order_release);
+  }
+  *sm_count = g_sm_count[dev].load(std::memory_order_relaxed);
+  return STAND_OK;
+}
+
+int launch_row_pass(const void* logits, long long rows, int V, int dtype, int n_chunks, float c, float2* pairs, int* status,
+                    cudaStream_t st) {
   RowPassParams rp;
-  rp.logits = logits; rp.rows = rows; rp.V = V; rp.n_chunks = n_chunks; rp.cpu = cpu; rp.upr = upr; rp.c = c;
-  rp.topk = topk; rp.pairs = pairs; rp.part = part;
-  const long long units = rows * upr;
-  const long long blocks = (units + K1_WARPS - 1) / K1_WARPS;
-  if (blocks <= 0 || blocks > 0x7FFFFFFFll) return STAND_E_ARG;
-  const bool al = rows_aligned(logits, V, dtype);
-  if (dtype == STAND_DTYPE_BF16) {
-    if (al) row_pass_kernel<1, true><<<(unsigned)blocks, K1_THREADS, 0, st>>>(rp);
-    else row_pass_kernel<1, false><<<(unsigned)blocks, K1_THREADS, 0, st>>>(rp);
+  rp.logits = logits; rp.rows = rows; rp.V = V; rp.n_chunks = n_chunks; rp.c = c; rp.pairs = pairs; rp.status = status;
+  rp.tiles_per_row = (n_chunks + TILE_CHUNKS - 1) / TILE_CHUNKS;
+  rp.total_tiles = rows * rp.tiles_per_row;
+  if (rows <= 0 || rows * n_chunks > 0x7FFFFFFFll * 8) return STAND_E_ARG;
+  if (rows_aligned(logits, V, dtype)) {
+    int sms = 0;
+    const int rc = prepare_device(&sms);
+    if (rc) return rc;
+    const long long want = 2ll * sms;  // two CTAs per SM, each walks a contiguous range of tiles
+    const unsigned grid = (unsigned)(rp.total_tiles < want ? rp.total_tiles : want);
+    if (dtype == STAND_DTYPE_BF16) row_pass_kernel<1><<<grid, K1_THREADS, K1_SMEM_DATA, st>>>(rp);
+    else row_pass_kernel<0><<<grid, K1_THREADS, K1_SMEM_DATA, st>>>(rp);
   } else {
-    if (al) row_pass_kernel<0, true><<<(unsigned)blocks, K1_THREADS, 0, st>>>(rp);
-    else row_pass_kernel<0, false><<<(unsigned)blocks, K1_THREADS, 0, st>>>(rp);
+    const unsigned blocks = (unsigned)((rows * n_chunks + 7) / 8);
+    if (dtype == STAND_DTYPE_BF16) row_pass_plain_kernel<1><<<blocks, 256, 0, st>>>(rp);
+    else row_pass_plain_kernel<0><<<blocks, 256, 0, st>>>(rp);
   }
   return launch_ok();
 }
@@ -163,17 +179,17 @@ int launch_row_pass(const void* logits, long long rows, int V, int dtype, int n_
 int run_verify(stand_ctx* x, const void* logits, int32_t* emitted, int32_t* n_emitted, cudaStream_t st) {
   const stand_config& c = x->cfg;
   if (x->ev_before) cudaEventRecord(x->ev_before, st);
-  int rc = launch_row_pass(logits, (long long)c.B * c.N, c.V, c.dtype, x->d.n_chunks, x->d.cpu, x->d.upr, x->c, c.topk,
-                           x->at<float2>(x->L.pairs), x->at<uint2>(x->L.part), st);
+  int rc = launch_row_pass(logits, (long long)c.B * c.N, c.V, c.dtype, x->d.n_chunks, x->c, x->at<float2>(x->L.pairs),
+                           x->at<int>(x->L.status), st);
   if (rc) return rc;
   if (x->ev_after) cudaEventRecord(x->ev_after, st);
   x->launches += 1;
   x->step += 1;  // the tree drafted in step s-1 is verified in step s
   VerifyParams v;
   v.logits = logits; v.dtype = c.dtype; v.B = c.B; v.N = c.N; v.V = c.V; v.K = c.topk; v.n_max = c.order_max;
-  v.D = x->d.D; v.n_chunks = x->d.n_chunks; v.upr = x->d.upr; v.c = x->c; v.seed = c.seed; v.step = x->step;
+  v.D = x->d.D; v.n_chunks = x->d.n_chunks; v.c = x->c; v.seed = c.seed; v.step = x->step;
   v.first_child = x->topo_first_child(); v.n_children = x->topo_n_children();
-  v.pairs = x->at<float2>(x->L.pairs); v.part = x->at<uint2>(x->L.part);
+  v.pairs = x->at<float2>(x->L.pairs);
   v.tail = x->at<int>(x->L.tail); v.len = x->at<long long>(x->L.len); v.tree = x->at<int>(x->L.tree);
   v.cand_n = x->at<int>(x->L.cand_n); v.cand_id = x->at<int>(x->L.cand_id); v.cand_phi = x->at<float>(x->L.cand_phi);
   v.emitted_user = emitted; v.n_emitted_user = n_emitted;
@@ -399,8 +415,8 @@ size_t stand_row_stats_scratch_bytes(int64_t rows, int32_t V, int32_t dtype, int
   if (rows < 1 || V < 2 || V > STAND_MAX_VOCAB || topk < 1 || topk > STAND_MAX_TOPK) return 0;
   if (dtype != STAND_DTYPE_F32 && dtype != STAND_DTYPE_BF16) return 0;
   const size_t n_chunks = (V + CHUNK - 1) / CHUNK;
-  // one unit per chunk at most
-  return align_up((size_t)rows * n_chunks * sizeof(float2)) + align_up((size_t)rows * n_chunks * topk * sizeof(uint2));
+  // a status word, then one (sum, max) pair per chunk
+  return 256 + align_up((size_t)rows * n_chunks * sizeof(float2));
 }
 
 int stand_row_stats(const void* dev_logits, int64_t rows, int32_t V, int32_t dtype, float temperature, int32_t topk,
@@ -411,19 +427,17 @@ int stand_row_stats(const void* dev_logits, int64_t rows, int32_t V, int32_t dty
   if (!dev_scratch || ((uintptr_t)dev_scratch & 255) != 0 || scratch_bytes < need) return STAND_E_WORKSPACE;
   cudaStream_t st = (cudaStream_t)cu_stream;
   const int n_chunks = (V + CHUNK - 1) / CHUNK;
-  long long cpu = ((long long)rows * n_chunks + 7103) / 7104;
-  if (cpu < 1) cpu = 1;
-  if (cpu > n_chunks) cpu = n_chunks;
-  const int upr = (int)((n_chunks + cpu - 1) / cpu);
-  float2* pairs = (float2*)dev_scratch;
-  uint2* part = (uint2*)((char*)dev_scratch + align_up((size_t)rows * n_chunks * sizeof(float2)));
+  int* status = (int*)dev_scratch;
+  float2* pairs = (float2*)((char*)dev_scratch + 256);
   const float c = log2e_over_T(temperature);
-  int rc = launch_row_pass(dev_logits, rows, V, dtype, n_chunks, (int)cpu, upr, c, topk, pairs, part, st);
+  int rc = cuda_ok(cudaMemsetAsync(status, 0, sizeof(int), st));  // the scratch may hold an earlier call's status
+  if (rc) return rc;
+  rc = launch_row_pass(dev_logits, rows, V, dtype, n_chunks, c, pairs, status, st);
   if (rc) return rc;
   RowFinalizeParams f;
-  f.pairs = pairs; f.part = part; f.rows = rows; f.n_chunks = n_chunks; f.upr = upr; f.topk = topk; f.c = c;
-  f.lse = dev_lse; f.ids = dev_ids; f.values = dev_values; f.probs = dev_probs;
-  row_finalize_kernel<<<(unsigned)((rows + 7) / 8), 256, 0, st>>>(f);
+  f.logits = dev_logits; f.dtype = dtype; f.V = V; f.pairs = pairs; f.status = status; f.rows = rows; f.n_chunks = n_chunks;
+  f.topk = topk; f.c = c; f.lse = dev_lse; f.ids = dev_ids; f.values = dev_values; f.probs = dev_probs;
+  row_finalize_kernel<<<(unsigned)((rows + FIN_WARPS - 1) / FIN_WARPS), FIN_WARPS * 32, 0, st>>>(f);
   return launch_ok();
 }
 
@@ -468,6 +482,10 @@ int stand_get_stats(stand_ctx* x, stand_stats* host_out) {
   host_out->lookups = s[ST_LOOKUPS];
   for (int i = 0; i < STAND_MAX_ORDER; ++i) host_out->lookup_hits[i] = s[ST_HIT0 + i];
   host_out->max_probe_seen = s[ST_MAX_PROBE];
+  int status = 0;
+  rc = cuda_ok(cudaMemcpy(&status, x->ws + x->L.status, sizeof(int), cudaMemcpyDeviceToHost));
+  if (rc) return rc;
+  host_out->wait_timeouts = (uint64_t)(status != 0);
   return STAND_OK;
 }
 

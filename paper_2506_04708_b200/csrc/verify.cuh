@@ -10,8 +10,10 @@
 //                        by a running factor, so the residual needs no pass over V;
 //   phase 3 (all warps)  the one sampled token: inverse CDF in token order, coarse
 //                        over chunk masses, then exact inside one 1024-entry chunk;
-//   phase 4              the accepted rows compressed to top-k probabilities and the
-//                        context windows for the N-gram update; sequence tails advance.
+//   phase 4              the accepted rows compressed to top-k probabilities (the exact
+//                        top-k is finished here, from the few chunks whose maximum
+//                        can reach it) and the context windows for the N-gram
+//                        update; sequence tails advance.
 // Decisions are taken in double precision on top of the row pass's fp32 chunk sums.
 #pragma once
 #include "common.cuh"
@@ -23,14 +25,13 @@ constexpr int K2_THREADS = 256;
 
 struct VerifyParams {
   const void* logits;
-  int dtype, B, N, V, K, n_max, D, n_chunks, upr;
+  int dtype, B, N, V, K, n_max, D, n_chunks;
   float c;
   unsigned long long seed;
   uint32_t step;
   const int* first_child;  // [N]
   const int* n_children;   // [N]
-  const float2* pairs;     // [B*N, n_chunks]
-  const uint2* part;       // [B*N, upr, K]
+  const float2* pairs;     // [B*N, n_chunks] (sum, chunk max) from the row pass
   int* tail;               // [B, n_max]   advanced here
   long long* len;          // [B]          advanced here
   const int* tree;         // [B, N]
@@ -87,6 +88,8 @@ __global__ void __launch_bounds__(K2_THREADS) verify_kernel(const VerifyParams p
   __shared__ double s_scale;         // residual target off the candidates = scale * target
   __shared__ int s_pick, s_pick_last;
   __shared__ double s_base;
+  __shared__ uint2 s_buf[K2_THREADS / 32][CAND_CAP];  // per-warp candidate buffers of the top-k selection
+  __shared__ int s_cnt[K2_THREADS / 32];
 
   const int b = blockIdx.x;
   const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
@@ -96,7 +99,7 @@ __global__ void __launch_bounds__(K2_THREADS) verify_kernel(const VerifyParams p
   // ---- phase 1 -----------------------------------------------------------
   for (int u = warp; u < N; u += K2_THREADS / 32) {
     const long long row = (long long)b * N + u;
-    const RowNorm nm = row_normaliser(p.pairs + row * p.n_chunks, p.n_chunks, lane);
+    const RowNorm nm = row_normaliser(p.pairs + row * p.n_chunks, p.n_chunks, p.c, lane);
     if (lane == 0) { s_off[u] = nm.off; s_Z[u] = nm.Z; }
     const int nc = p.cand_n[row];
     if (lane < nc) {
@@ -191,7 +194,7 @@ __global__ void __launch_bounds__(K2_THREADS) verify_kernel(const VerifyParams p
     const int ch = tid * per + i;
     if (i < per && ch < p.n_chunks) {
       const float2 pr = p.pairs[rows * p.n_chunks + ch];
-      double mass = pr.x > 0.0f ? scale * ((double)pr.x * exp2((double)pr.y - (double)off) / Z) : 0.0;
+      double mass = scale * (chunk_mass(pr, p.c, off) / Z);
       for (int s = 0; s < nsup; ++s)
         if (s_sup_id[s] / CHUNK == ch) mass += s_sup_pt[s] - scale * s_sup_p[s];
       cm[i] = fmax(mass, 0.0);
@@ -294,26 +297,26 @@ __global__ void __launch_bounds__(K2_THREADS) verify_kernel(const VerifyParams p
     if (p.emitted_user) p.emitted_user[b * W1 + tid] = e;
     p.path[b * W1 + tid] = tid <= m ? s_path[tid] : -1;
   }
-  // compressed rows of the accepted path: merge the unit lists, convert to probabilities
+  // compressed rows of the accepted path: the exact top-k of each row, as probabilities
   for (int j = warp; j <= m; j += K2_THREADS / 32) {
     const int u = s_path[j];
     const long long row = (long long)b * N + u;
-    const uint2* part = p.part + row * p.upr * K;
     const float o = s_off[u];
     const double z = s_Z[u];
-    unsigned long long below = ~0ull;
-    for (int r = 0; r < K; ++r) {
-      const unsigned long long key = next_best(part, p.upr * K, below, lane);
-      if (lane == 0) {
-        const long long at = ((long long)b * W1 + j) * K + r;
-        if (key == 0ull) { p.rec_ids[at] = -1; p.rec_p[at] = 0.0f; }
-        else {
-          p.rec_ids[at] = (int)key_id(key);
-          p.rec_p[at] = (float)(exp2((double)key_value(key) * cd - (double)o) / z);
-        }
+    const int n = row_topk_warp(p.logits, p.dtype, row, p.V, p.pairs + row * p.n_chunks, p.n_chunks, K, s_buf[warp],
+                                &s_cnt[warp], lane);
+    if (lane < K) {
+      const long long at = ((long long)b * W1 + j) * K + lane;
+      if (lane < n) {
+        const uint2 e = s_buf[warp][lane];
+        p.rec_ids[at] = (int)e.y;
+        p.rec_p[at] = (float)(exp2((double)__uint_as_float(e.x) * cd - (double)o) / z);
+      } else {
+        p.rec_ids[at] = -1;
+        p.rec_p[at] = 0.0f;
       }
-      below = key;
     }
+    __syncwarp();
   }
 }
 

@@ -52,7 +52,7 @@ def test_static_scratch_matches_caller_scratch_twice_in_a_row(dtype):
 def test_static_scratch_refuses_what_does_not_fit():
     import torch
     from paper_2506_04708_b200 import binding
-    rows, V, k = 4096, 151936, 10
+    rows, V, k = 8192, 151936, 10
     assert binding.lib().stand_row_stats_scratch_bytes(rows, V, binding.DTYPE_BF16, k) > binding.STATIC_SCRATCH_BYTES
     # the refusal comes before any launch, so the logits are never read: a small tensor stands in
     dl = torch.zeros((rows, 8), dtype=torch.bfloat16, device="cuda:0")
