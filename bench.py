@@ -110,11 +110,19 @@ def pregrow(gpu, w, seed, torch):
     return gpu.stats()["inserts"]
 
 
+def workload_of(args):
+    """The named workload; --batch scales the number of sequences (for profiling a smaller case of the same kernels)."""
+    w = inputs.WORKLOADS[args.workload]
+    if args.batch:
+        w = inputs.scaled(w, name=f"{w.name}@B={args.batch}", B=args.batch)
+    return w
+
+
 def run_ours(args, rank, world, local):
     import torch
     from paper_2506_04708_b200.binding import Stand
 
-    w = inputs.WORKLOADS[args.workload]
+    w = workload_of(args)
     dev = torch.device("cuda", local)
     torch.cuda.set_device(dev)
     dist = None
@@ -130,6 +138,8 @@ def run_ours(args, rank, world, local):
     while ring_n * step_bytes < 3 * L2_BYTES:
         ring_n += 1
     ring_n = min(ring_n, 64)
+    if args.ring:
+        ring_n = args.ring
 
     gpu = Stand(w.B, w.N, w.V, w.topk, w.order_max, w.dtype, w.T, seed, w.table_slots, parent, device=dev,
                 host_staging=True)
@@ -311,7 +321,7 @@ def run_reference(args, rank, world):
     """The oracle as it stands, on the host cores: the reference arm."""
     if rank != 0:
         return
-    w = inputs.WORKLOADS[args.workload]
+    w = workload_of(args)
     r = time_oracle(w, None, args, total_budget_s=90.0, steps=args.steps, warmup=args.warmup)
     line = {"impl": "reference", "metric": METRIC, "value": r["value"], "unit": UNIT, "n_gpus": world,
             "steps": args.steps, "warmup": args.warmup, "ms_per_step": r["ms_per_step"], "higher_is_better": True,
@@ -334,6 +344,8 @@ def main():
     ap.add_argument("--peak-mode", default="add8", choices=["add8", "p80"])
     ap.add_argument("--seed", type=int, default=0)
     ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--batch", type=int, default=0, help="override the workload's number of sequences (profiling)")
+    ap.add_argument("--ring", type=int, default=0, help="override the number of logit buffers in the ring (profiling)")
     args = ap.parse_args()
     rank = int(os.environ.get("RANK", "0"))
     world = int(os.environ.get("WORLD_SIZE", "1"))

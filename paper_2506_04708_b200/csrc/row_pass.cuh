@@ -10,21 +10,23 @@
 // the few rows that need it (row_topk_warp below).
 //
 // The kernel is bound by HBM bandwidth: persistent CTAs (two per SM) walk a
-// contiguous range of 8-chunk tiles; one elected lane streams tiles into a ring of
-// shared-memory stages with bulk asynchronous copies (TMA) that complete on
-// mbarriers, marked evict-first in L2; eight consumer warps take one chunk of a
-// tile each.  The inner loop has no branches: packed bf16 max, packed fp32 FMA/ADD,
+// contiguous range of tiles (16 chunks for bf16, 8 for fp32); one elected lane
+// streams tiles into a ring of shared-memory stages with bulk asynchronous copies
+// (TMA) that complete on mbarriers, marked evict-first in L2; each consumer warp
+// takes one chunk of every tile.  The inner loop has no branches: packed bf16 max, packed fp32 FMA/ADD,
 // one ex2 per entry.
 #pragma once
 #include "common.cuh"
 
 namespace stand {
 
-constexpr int K1_CONSUMER_WARPS = 8;                       // = chunks per tile
-constexpr int K1_THREADS = (K1_CONSUMER_WARPS + 1) * 32;   // + the producer warp
-constexpr int TILE_CHUNKS = K1_CONSUMER_WARPS;
-constexpr int TILE_ELEMS = TILE_CHUNKS * CHUNK;
-constexpr int K1_SMEM_DATA = 96 * 1024;                    // ring bytes per CTA (two CTAs per SM)
+constexpr int K1_SMEM_DATA = 96 * 1024;  // ring bytes per CTA at two CTAs per SM
+constexpr int K1_CTAS = 2;               // persistent CTAs per SM
+// consumer warps per CTA = chunks per tile: bf16 needs 32 warps per SM to keep the exp unit fed (16 per CTA:
+// 6.6 TB/s against 6.2 TB/s with 8); fp32 moves twice the bytes per exp and is fed by 8.
+template <int DT> struct K1Shape { static constexpr int CW = DT == 1 ? 16 : 8; };
+template <int DT> constexpr int k1_stage_bytes() { return K1Shape<DT>::CW * CHUNK * (DT == 1 ? 2 : 4); }
+template <int DT> constexpr int k1_smem_bytes() { return (K1_SMEM_DATA / k1_stage_bytes<DT>()) * k1_stage_bytes<DT>(); }
 constexpr unsigned SPIN_LIMIT = 1u << 22;                  // bounded waits: about a second, then the kernel gives up
 
 constexpr int COMPACT_AT = 64;              // candidate count that triggers a compaction
@@ -106,6 +108,10 @@ template <> struct ElemTraits<0> {  // float
     sum2 = add2(sum2, pack2(ex2_approx(a), ex2_approx(b)));
     unpack2(fma2(pack2(__uint_as_float(d.z), __uint_as_float(d.w)), c2, no2), a, b);
     sum2 = add2(sum2, pack2(ex2_approx(a), ex2_approx(b)));
+  }
+  __device__ static __forceinline__ void unpack(const uint4& d, float (&f)[4]) {
+    f[0] = __uint_as_float(d.x); f[1] = __uint_as_float(d.y);
+    f[2] = __uint_as_float(d.z); f[3] = __uint_as_float(d.w);
   }
 };
 template <> struct ElemTraits<1> {  // bfloat16, two per word, lower index in the low half
@@ -210,12 +216,12 @@ __device__ __forceinline__ void bulk_load(uint32_t dst, const void* src, uint32_
 // The streaming kernel.  Requires a 16-byte aligned base and V * sizeof(elem) a
 // multiple of 16 (the host checks and falls back to row_pass_plain_kernel).
 // ---------------------------------------------------------------------------------
-template <int DT>
-__global__ void __launch_bounds__(K1_THREADS, 2) row_pass_kernel(const RowPassParams p) {
+template <int DT, int CW, int CTAS>  // CW consumer warps = chunks per tile; CTAS CTAs per SM share the ring budget
+__global__ void __launch_bounds__((CW + 1) * 32, CTAS) row_pass_kernel(const RowPassParams p) {
   using TR = ElemTraits<DT>;
   constexpr int VEC = TR::VEC, NV = CHUNK / (32 * VEC);
-  constexpr int STAGE_BYTES = TILE_ELEMS * TR::ESIZE;
-  constexpr int STAGES = K1_SMEM_DATA / STAGE_BYTES;
+  constexpr int STAGE_BYTES = CW * CHUNK * TR::ESIZE;
+  constexpr int STAGES = (2 * K1_SMEM_DATA / CTAS) / STAGE_BYTES;
   static_assert(STAGES >= 2, "ring too small");
   extern __shared__ __align__(128) unsigned char smem[];
   __shared__ __align__(8) unsigned long long s_full[STAGES], s_empty[STAGES];
@@ -224,46 +230,47 @@ __global__ void __launch_bounds__(K1_THREADS, 2) row_pass_kernel(const RowPassPa
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   const long long t0 = (long long)blockIdx.x * p.total_tiles / gridDim.x;
   const long long t1 = (long long)(blockIdx.x + 1) * p.total_tiles / gridDim.x;
-  const long long n_tiles = t1 - t0;
+  const int n_tiles = (int)(t1 - t0);
   if (threadIdx.x == 0) {
     s_abort = 0;
     for (int s = 0; s < STAGES; ++s) {
       mbar_init(smem_addr(&s_full[s]), 1);
-      mbar_init(smem_addr(&s_empty[s]), K1_CONSUMER_WARPS);
+      mbar_init(smem_addr(&s_empty[s]), CW);
     }
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
   }
   __syncthreads();
   const size_t row_bytes = (size_t)p.V * TR::ESIZE;
+  // tile coordinates advance without divisions
+  long long row = t0 / p.tiles_per_row;
+  int t = (int)(t0 - row * p.tiles_per_row);
 
-  if (warp == K1_CONSUMER_WARPS) {
+  if (warp == CW) {
     // ---- producer: one lane keeps the ring full ------------------------------------
     if (lane == 0) {
       const unsigned long long policy = l2_evict_first_policy();
-      long long issued = 0;
-      for (long long i = 0; i < n_tiles; ++i) {
-        const int s = (int)(i % STAGES);
-        const uint32_t round = (uint32_t)(i / STAGES);
-        if (!mbar_wait_bounded(smem_addr(&s_empty[s]), (round & 1u) ^ 1u, &s_abort)) {
+      int issued = 0, s = 0;
+      uint32_t parity = 1;  // waiting for the phase before the first one succeeds at once
+      const char* src_row = (const char*)p.logits + (size_t)row * row_bytes;
+      for (int i = 0; i < n_tiles; ++i) {
+        if (!mbar_wait_bounded(smem_addr(&s_empty[s]), parity, &s_abort)) {
           if (!s_abort && p.status) atomicExch(p.status, K1_ERR_EMPTY_WAIT);
           s_abort = 1;
           break;
         }
-        const long long g = t0 + i;
-        const long long row = g / p.tiles_per_row;
-        const int t = (int)(g - row * p.tiles_per_row);
         const size_t at = (size_t)t * STAGE_BYTES;
         const uint32_t bytes = (uint32_t)(row_bytes - at < (size_t)STAGE_BYTES ? row_bytes - at : (size_t)STAGE_BYTES);
         const uint32_t bar = smem_addr(&s_full[s]);
         mbar_expect_tx(bar, bytes);
-        bulk_load(smem_addr(smem + (size_t)s * STAGE_BYTES), (const char*)p.logits + (size_t)row * row_bytes + at, bytes, bar,
-                  policy);
+        bulk_load(smem_addr(smem + (size_t)s * STAGE_BYTES), src_row + at, bytes, bar, policy);
         issued = i + 1;
+        if (++t == p.tiles_per_row) { t = 0; src_row += row_bytes; }
+        if (++s == STAGES) { s = 0; parity ^= 1u; }
       }
       if (s_abort) {
         // leave no copy in flight behind: wait (bounded) for the stages that were issued last
-        for (long long i = issued > STAGES ? issued - STAGES : 0; i < issued; ++i) {
-          const uint32_t bar = smem_addr(&s_full[(int)(i % STAGES)]);
+        for (int i = issued > STAGES ? issued - STAGES : 0; i < issued; ++i) {
+          const uint32_t bar = smem_addr(&s_full[i % STAGES]);
           for (unsigned spin = 0; spin < SPIN_LIMIT && !mbar_try_wait(bar, (uint32_t)(i / STAGES) & 1u); ++spin) {}
         }
       }
@@ -273,10 +280,11 @@ __global__ void __launch_bounds__(K1_THREADS, 2) row_pass_kernel(const RowPassPa
 
   // ---- consumers: warp w takes chunk w of every tile -----------------------------------
   const float c = p.c;
-  for (long long i = 0; i < n_tiles; ++i) {
-    const int s = (int)(i % STAGES);
-    const uint32_t round = (uint32_t)(i / STAGES);
-    const bool landed = mbar_wait_bounded(smem_addr(&s_full[s]), round & 1u, &s_abort);
+  int s = 0;
+  uint32_t parity = 0;
+  float2* out = p.pairs + row * p.n_chunks;
+  for (int i = 0; i < n_tiles; ++i) {
+    const bool landed = mbar_wait_bounded(smem_addr(&s_full[s]), parity, &s_abort);
     if (!__all_sync(FULL, landed)) {  // warp-uniform: the lanes leave together
       if (lane == 0) {
         if (!s_abort && p.status) atomicExch(p.status, K1_ERR_FULL_WAIT);
@@ -284,10 +292,7 @@ __global__ void __launch_bounds__(K1_THREADS, 2) row_pass_kernel(const RowPassPa
       }
       break;
     }
-    const long long g = t0 + i;
-    const long long row = g / p.tiles_per_row;
-    const int t = (int)(g - row * p.tiles_per_row);
-    const int chunk = t * TILE_CHUNKS + warp;
+    const int chunk = t * CW + warp;
     if (chunk < p.n_chunks) {
       const uint4* src = reinterpret_cast<const uint4*>(smem + (size_t)s * STAGE_BYTES + (size_t)warp * CHUNK * TR::ESIZE);
       uint4 v[NV];
@@ -302,10 +307,12 @@ __global__ void __launch_bounds__(K1_THREADS, 2) row_pass_kernel(const RowPassPa
       __syncwarp();
       if (lane == 0) mbar_arrive(smem_addr(&s_empty[s]));  // the data is in registers: hand the stage back early
       const float2 r = reduce_chunk<DT, NV>(v, c);
-      if (lane == 0) p.pairs[row * p.n_chunks + chunk] = r;
+      if (lane == 0) out[chunk] = r;
     } else {
       if (lane == 0) mbar_arrive(smem_addr(&s_empty[s]));
     }
+    if (++t == p.tiles_per_row) { t = 0; out += p.n_chunks; }
+    if (++s == STAGES) { s = 0; parity ^= 1u; }
   }
 }
 

@@ -142,9 +142,11 @@ int prepare_device(int* sm_count) {
   if (!g_k1_ready[dev].load(std::memory_order_acquire)) {
     int sms = 0;
     if (cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess || sms < 1) return STAND_E_CUDA;
-    if (cudaFuncSetAttribute(row_pass_kernel<0>, cudaFuncAttributeMaxDynamicSharedMemorySize, K1_SMEM_DATA) != cudaSuccess)
+    if (cudaFuncSetAttribute(row_pass_kernel<0, K1Shape<0>::CW, K1_CTAS>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                             k1_smem_bytes<0>()) != cudaSuccess)
       return STAND_E_CUDA;
-    if (cudaFuncSetAttribute(row_pass_kernel<1>, cudaFuncAttributeMaxDynamicSharedMemorySize, K1_SMEM_DATA) != cudaSuccess)
+    if (cudaFuncSetAttribute(row_pass_kernel<1, K1Shape<1>::CW, K1_CTAS>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                             k1_smem_bytes<1>()) != cudaSuccess)
       return STAND_E_CUDA;
     g_sm_count[dev].store(sms, std::memory_order_relaxed);
     g_k1_ready[dev].store(1, std::memory_order_release);
@@ -157,17 +159,20 @@ int launch_row_pass(const void* logits, long long rows, int V, int dtype, int n_
                     cudaStream_t st) {
   RowPassParams rp;
   rp.logits = logits; rp.rows = rows; rp.V = V; rp.n_chunks = n_chunks; rp.c = c; rp.pairs = pairs; rp.status = status;
-  rp.tiles_per_row = (n_chunks + TILE_CHUNKS - 1) / TILE_CHUNKS;
+  const int tile_chunks = dtype == STAND_DTYPE_BF16 ? K1Shape<1>::CW : K1Shape<0>::CW;
+  rp.tiles_per_row = (n_chunks + tile_chunks - 1) / tile_chunks;
   rp.total_tiles = rows * rp.tiles_per_row;
   if (rows <= 0 || rows * n_chunks > 0x7FFFFFFFll * 8) return STAND_E_ARG;
   if (rows_aligned(logits, V, dtype)) {
     int sms = 0;
     const int rc = prepare_device(&sms);
     if (rc) return rc;
-    const long long want = 2ll * sms;  // two CTAs per SM, each walks a contiguous range of tiles
+    const long long want = (long long)K1_CTAS * sms;  // each CTA walks a contiguous range of tiles
     const unsigned grid = (unsigned)(rp.total_tiles < want ? rp.total_tiles : want);
-    if (dtype == STAND_DTYPE_BF16) row_pass_kernel<1><<<grid, K1_THREADS, K1_SMEM_DATA, st>>>(rp);
-    else row_pass_kernel<0><<<grid, K1_THREADS, K1_SMEM_DATA, st>>>(rp);
+    if (dtype == STAND_DTYPE_BF16)
+      row_pass_kernel<1, K1Shape<1>::CW, K1_CTAS><<<grid, (K1Shape<1>::CW + 1) * 32, k1_smem_bytes<1>(), st>>>(rp);
+    else
+      row_pass_kernel<0, K1Shape<0>::CW, K1_CTAS><<<grid, (K1Shape<0>::CW + 1) * 32, k1_smem_bytes<0>(), st>>>(rp);
   } else {
     const unsigned blocks = (unsigned)((rows * n_chunks + 7) / 8);
     if (dtype == STAND_DTYPE_BF16) row_pass_plain_kernel<1><<<blocks, 256, 0, st>>>(rp);
