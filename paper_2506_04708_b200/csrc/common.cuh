@@ -12,6 +12,7 @@ constexpr int KMAX = 12;     // STAND_MAX_TOPK
 constexpr int ORDER_MAX = 4; // STAND_MAX_ORDER
 constexpr int NODES_MAX = 128;
 constexpr int DEPTH_MAX = 32;
+constexpr int VOCAB_MAX = 1 << 20;  // STAND_MAX_VOCAB
 
 constexpr uint32_t SLOT_FINAL = 0x40000000u;
 constexpr uint32_t SLOT_GUMBEL = 0x80000000u;

@@ -36,18 +36,27 @@ struct DraftParams {
 };
 
 __global__ void __launch_bounds__(K4_THREADS) draft_kernel(const DraftParams p) {
-  __shared__ int s_tok[NODES_MAX];
+  __shared__ int s_tok[NODES_MAX], s_parent[NODES_MAX], s_fc[NODES_MAX], s_nch[NODES_MAX];
+  __shared__ int s_tail[ORDER_MAX], s_level[DEPTH_MAX + 2];
   const int b = blockIdx.x, tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
   const int N = p.N, K = p.K, n_max = p.n_max;
-  for (int u = tid; u < N; u += K4_THREADS) s_tok[u] = -1;
+  // topology and tail once, with coalesced loads: the level loop below touches shared memory only
+  for (int u = tid; u < N; u += K4_THREADS) {
+    s_tok[u] = -1;
+    s_parent[u] = p.parent[u];
+    s_fc[u] = p.first_child[u];
+    s_nch[u] = p.n_children[u];
+  }
+  if (tid < n_max) s_tail[tid] = p.tail[b * n_max + tid];
+  if (tid <= p.D + 1) s_level[tid] = p.level_start[tid];
   __syncthreads();
-  if (tid == 0) s_tok[0] = p.tail[b * n_max + n_max - 1];  // the root carries the last token
+  if (tid == 0) s_tok[0] = s_tail[n_max - 1];  // the root carries the last token
   __syncthreads();
 
   for (int d = 0; d < p.D; ++d) {
-    const int l0 = p.level_start[d], l1 = p.level_start[d + 1];
+    const int l0 = s_level[d], l1 = s_level[d + 1];
     for (int u = l0 + warp; u < l1; u += K4_THREADS / 32) {
-      const int m = p.n_children[u];
+      const int m = s_nch[u];
       const long long row = (long long)b * N + u;
       if (m == 0) { if (lane == 0) p.cand_n[row] = 0; continue; }
       const bool drafted = u == 0 || s_tok[u] >= 0;
@@ -56,8 +65,8 @@ __global__ void __launch_bounds__(K4_THREADS) draft_kernel(const DraftParams p) 
       int win[ORDER_MAX];
       {
         int filled = 0, w = u;
-        while (w != 0 && filled < n_max) { win[n_max - 1 - filled] = s_tok[w]; ++filled; w = p.parent[w]; }
-        for (int i = n_max - 1; filled < n_max; --i, ++filled) win[n_max - 1 - filled] = p.tail[b * n_max + i];
+        while (w != 0 && filled < n_max) { win[n_max - 1 - filled] = s_tok[w]; ++filled; w = s_parent[w]; }
+        for (int i = n_max - 1; filled < n_max; --i, ++filled) win[n_max - 1 - filled] = s_tail[i];
       }
       // one group of 8 lanes per order: all orders are probed at once
       const int grp = lane / GROUP;
@@ -101,7 +110,7 @@ __global__ void __launch_bounds__(K4_THREADS) draft_kernel(const DraftParams p) 
         const bool vj = __shfl_sync(FULL, (int)valid, j) != 0;
         if (vj && (gj > g || (gj == g && idj < id))) ++rank;
       }
-      if (valid && rank < m) s_tok[p.first_child[u] + rank] = id;
+      if (valid && rank < m) s_tok[s_fc[u] + rank] = id;
       const unsigned vmask = __ballot_sync(FULL, valid);
       if (valid) {
         const int pos = __popc(vmask & ((1u << lane) - 1u));
@@ -113,7 +122,7 @@ __global__ void __launch_bounds__(K4_THREADS) draft_kernel(const DraftParams p) 
     __syncthreads();
   }
   // nodes of the deepest level have no children
-  for (int u = p.level_start[p.D] + tid; u < N; u += K4_THREADS) p.cand_n[(long long)b * N + u] = 0;
+  for (int u = s_level[p.D] + tid; u < N; u += K4_THREADS) p.cand_n[(long long)b * N + u] = 0;
   for (int u = tid; u < N; u += K4_THREADS) {
     const int t = s_tok[u];
     p.tree[(long long)b * N + u] = t;

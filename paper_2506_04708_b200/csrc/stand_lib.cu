@@ -104,6 +104,7 @@ struct stand_ctx {
   char* ws;
   uint32_t step;
   bool pending;
+  bool located;  // the pending verification already mapped its records to slots
   uint64_t launches;
   cudaStream_t last_stream;
   int max_probe;
@@ -181,7 +182,24 @@ int launch_row_pass(const void* logits, long long rows, int V, int dtype, int n_
   return launch_ok();
 }
 
-int run_verify(stand_ctx* x, const void* logits, int32_t* emitted, int32_t* n_emitted, cudaStream_t st) {
+UpdateParams update_params(stand_ctx* x, long long n_rows, const int* ctxw, const int* ids, const float* probs,
+                           const int* n_path, int width) {
+  const stand_config& c = x->cfg;
+  UpdateParams u;
+  u.table = x->at<Slot>(x->L.table); u.mask = c.table_slots - 1; u.max_probe = x->max_probe; u.V = c.V; u.K = c.topk;
+  u.n_max = c.order_max; u.n_rows = n_rows; u.rec_ctx = ctxw; u.rec_ids = ids; u.rec_p = probs; u.n_path = n_path;
+  u.width = width; u.rec_slot = x->at<uint32_t>(x->L.rec_slot); u.stats = x->at<unsigned long long>(x->L.stats);
+  return u;
+}
+
+UpdateParams step_update_params(stand_ctx* x) {
+  const int W = x->d.D + 1;
+  return update_params(x, (long long)x->cfg.B * W, x->at<int>(x->L.rec_ctx), x->at<int>(x->L.rec_ids),
+                       x->at<float>(x->L.rec_p), x->at<int>(x->L.n_path), W);
+}
+
+// fuse_locate: the verification kernel also maps this step's records to table slots (stage 1 of the update).
+int run_verify(stand_ctx* x, const void* logits, int32_t* emitted, int32_t* n_emitted, bool fuse_locate, cudaStream_t st) {
   const stand_config& c = x->cfg;
   if (x->ev_before) cudaEventRecord(x->ev_before, st);
   int rc = launch_row_pass(logits, (long long)c.B * c.N, c.V, c.dtype, x->d.n_chunks, x->c, x->at<float2>(x->L.pairs),
@@ -201,38 +219,36 @@ int run_verify(stand_ctx* x, const void* logits, int32_t* emitted, int32_t* n_em
   v.emitted = x->at<int>(x->L.emitted); v.n_path = x->at<int>(x->L.n_path); v.path = x->at<int>(x->L.path);
   v.rec_ctx = x->at<int>(x->L.rec_ctx); v.rec_ids = x->at<int>(x->L.rec_ids); v.rec_p = x->at<float>(x->L.rec_p);
   v.stats = x->at<unsigned long long>(x->L.stats);
+  v.fuse_locate = fuse_locate ? 1 : 0;
+  v.upd = step_update_params(x);
   verify_kernel<<<c.B, K2_THREADS, 0, st>>>(v);
   rc = launch_ok();
   if (rc) return rc;
   x->launches += 1;
   x->pending = true;
+  x->located = fuse_locate;
   return STAND_OK;
 }
 
-int run_update_rows(stand_ctx* x, long long n_rows, const int* ctxw, const int* ids, const float* probs, const int* n_path,
-                    int width, cudaStream_t st) {
-  const stand_config& c = x->cfg;
-  UpdateParams u;
-  u.table = x->at<Slot>(x->L.table); u.mask = c.table_slots - 1; u.max_probe = x->max_probe; u.V = c.V; u.K = c.topk;
-  u.n_max = c.order_max; u.n_rows = n_rows; u.rec_ctx = ctxw; u.rec_ids = ids; u.rec_p = probs; u.n_path = n_path;
-  u.width = width; u.rec_slot = x->at<uint32_t>(x->L.rec_slot); u.stats = x->at<unsigned long long>(x->L.stats);
-  const long long n_rec = n_rows * c.order_max;
-  update_locate_kernel<<<(unsigned)((n_rec * GROUP + 255) / 256), 256, 0, st>>>(u);
-  int rc = launch_ok();
-  if (rc) return rc;
+int run_update_rows(stand_ctx* x, const UpdateParams& u, bool located, cudaStream_t st) {
+  const long long n_rec = u.n_rows * u.n_max;
+  int rc;
+  if (!located) {
+    update_locate_kernel<<<(unsigned)((n_rec * GROUP + 255) / 256), 256, 0, st>>>(u);
+    rc = launch_ok();
+    if (rc) return rc;
+    x->launches += 1;
+  }
   update_apply_kernel<<<(unsigned)((n_rec + APPLY_WARPS - 1) / APPLY_WARPS), APPLY_WARPS * 32, 0, st>>>(u);
   rc = launch_ok();
   if (rc) return rc;
-  x->launches += 2;
+  x->launches += 1;
   return STAND_OK;
 }
 
 int run_update(stand_ctx* x, cudaStream_t st) {
-  const stand_config& c = x->cfg;
-  const int W = x->d.D + 1;
-  const int rc = run_update_rows(x, (long long)c.B * W, x->at<int>(x->L.rec_ctx), x->at<int>(x->L.rec_ids),
-                                 x->at<float>(x->L.rec_p), x->at<int>(x->L.n_path), W, st);
-  if (rc == STAND_OK) x->pending = false;
+  const int rc = run_update_rows(x, step_update_params(x), x->located, st);
+  if (rc == STAND_OK) { x->pending = false; x->located = false; }
   return rc;
 }
 
@@ -288,6 +304,7 @@ int stand_init(const stand_config* cfg, void* dev_workspace, size_t bytes, stand
   x->ws = (char*)dev_workspace;
   x->step = 0;
   x->pending = false;
+  x->located = false;
   x->launches = 0;
   x->last_stream = 0;
   x->max_probe = cfg->max_probe > 0 ? cfg->max_probe : 96;
@@ -341,13 +358,15 @@ int stand_reset_sequences(stand_ctx* x, const int32_t* dev_tail, const int64_t* 
   if (rc) return rc;
   x->launches += 1;
   x->pending = false;
+  x->located = false;
   return STAND_OK;
 }
 
 int stand_verify_tree(stand_ctx* x, const void* dev_logits, int32_t* dev_emitted, int32_t* dev_n_emitted, void* cu_stream) {
   if (!x || !dev_logits) return STAND_E_ARG;
   x->last_stream = (cudaStream_t)cu_stream;
-  return run_verify(x, dev_logits, dev_emitted, dev_n_emitted, (cudaStream_t)cu_stream);
+  if (x->pending && x->located) return STAND_E_STATE;  // slots are marked for an update that has not run
+  return run_verify(x, dev_logits, dev_emitted, dev_n_emitted, false, (cudaStream_t)cu_stream);
 }
 
 int stand_ngram_update(stand_ctx* x, void* cu_stream) {
@@ -365,8 +384,8 @@ int stand_ngram_update_bulk(stand_ctx* x, const int32_t* dev_ctx, const int32_t*
   const stand_config& c = x->cfg;
   for (int64_t at = 0; at < M; at += BULK_ROWS) {
     const long long n = M - at < BULK_ROWS ? M - at : BULK_ROWS;
-    const int rc = run_update_rows(x, n, dev_ctx + at * c.order_max, dev_ids + at * c.topk, dev_probs + at * c.topk,
-                                   nullptr, 1, st);
+    const int rc = run_update_rows(x, update_params(x, n, dev_ctx + at * c.order_max, dev_ids + at * c.topk,
+                                                    dev_probs + at * c.topk, nullptr, 1), false, st);
     if (rc) return rc;
   }
   return STAND_OK;
@@ -383,7 +402,8 @@ int stand_step(stand_ctx* x, const void* dev_logits, int32_t* dev_emitted, int32
   if (!x || !dev_logits) return STAND_E_ARG;
   cudaStream_t st = (cudaStream_t)cu_stream;
   x->last_stream = st;
-  int rc = run_verify(x, dev_logits, dev_emitted, dev_n_emitted, st);
+  if (x->pending && x->located) return STAND_E_STATE;
+  int rc = run_verify(x, dev_logits, dev_emitted, dev_n_emitted, true, st);
   if (rc) return rc;
   rc = run_update(x, st);
   if (rc) return rc;
@@ -400,7 +420,7 @@ int stand_step_host(stand_ctx* x, const void* host_logits, int32_t* host_emitted
   const size_t bytes = (size_t)c.B * c.N * c.V * esize_of(c.dtype);
   int rc = cuda_ok(cudaMemcpyAsync(x->ws + x->L.staging, host_logits, bytes, cudaMemcpyHostToDevice, st));
   if (rc) return rc;
-  rc = run_verify(x, x->ws + x->L.staging, nullptr, nullptr, st);
+  rc = run_verify(x, x->ws + x->L.staging, nullptr, nullptr, true, st);
   if (rc) return rc;
   rc = run_update(x, st);
   if (rc) return rc;
@@ -587,7 +607,7 @@ int stand_state_load(stand_ctx* x, const int32_t* dev_tail, const int64_t* dev_l
   cp(x->L.cand_n, dev_cand_n, BN * 4);
   cp(x->L.cand_id, dev_cand_id, BN * c.topk * 4);
   cp(x->L.cand_phi, dev_cand_phi, BN * c.topk * 4);
-  if (rc == STAND_OK) { x->step = step; x->pending = false; }
+  if (rc == STAND_OK) { x->step = step; x->pending = false; x->located = false; }
   return rc;
 }
 

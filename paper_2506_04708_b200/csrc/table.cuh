@@ -322,15 +322,25 @@ __global__ void __launch_bounds__(APPLY_WARPS * 32) update_apply_kernel(const Up
   const bool fresh_slot = img->count == 0;
   merge_warp(img, p.rec_ids + row * p.K, p.rec_p + row * p.K, p.K, lane);
   uint32_t applied = 1;
-  for (long long i0 = (row + 1) & ~31ll; applied < pending && i0 < p.n_rows; i0 += 32) {
-    const long long i = i0 + lane;
-    const bool hit = i > row && i < p.n_rows && seg[i] == slot;
-    unsigned hits = __ballot_sync(FULL, hit);
-    while (hits) {
-      const int j = __ffs(hits) - 1;
-      hits &= hits - 1;
-      merge_warp(img, p.rec_ids + (i0 + j) * p.K, p.rec_p + (i0 + j) * p.K, p.K, lane);
-      ++applied;
+  // the other records of this slot, in row order; four 32-wide windows of rec_slot are in flight at once
+  constexpr int WIN = 4;
+  for (long long i0 = (row + 1) & ~31ll; applied < pending && i0 < p.n_rows; i0 += 32 * WIN) {
+    uint32_t got[WIN];
+#pragma unroll
+    for (int w = 0; w < WIN; ++w) {
+      const long long i = i0 + 32 * w + lane;
+      got[w] = (i > row && i < p.n_rows) ? seg[i] : NO_SLOT;
+    }
+#pragma unroll
+    for (int w = 0; w < WIN; ++w) {
+      unsigned hits = __ballot_sync(FULL, got[w] == slot);
+      while (hits) {
+        const int j = __ffs(hits) - 1;
+        hits &= hits - 1;
+        const long long i = i0 + 32 * w + j;
+        merge_warp(img, p.rec_ids + i * p.K, p.rec_p + i * p.K, p.K, lane);
+        ++applied;
+      }
     }
   }
   const int n_items = (int)img->n_items;

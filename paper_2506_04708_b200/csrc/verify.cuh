@@ -1,6 +1,8 @@
 // Verification walk (paper Sec. 3.2 speculative sampling, applied to the tree
 // drafted in Sec. 4.2).  One thread block per sequence.
 //
+//   phase 0 (all warps)  the sequence's tree, candidate lists and topology are staged in
+//                        shared memory with one round of coalesced loads;
 //   phase 1 (all warps)  normaliser of every row of the sequence from the chunk
 //                        pairs, and the target probability of every drafted
 //                        candidate (a handful of gathered logits per node);
@@ -13,11 +15,13 @@
 //   phase 4              the accepted rows compressed to top-k probabilities (the exact
 //                        top-k is finished here, from the few chunks whose maximum
 //                        can reach it) and the context windows for the N-gram
-//                        update; sequence tails advance.
+//                        update; sequence tails advance.  Optionally stage 1 of the
+//                        table update (context -> slot) for this sequence's records.
 // Decisions are taken in double precision on top of the row pass's fp32 chunk sums.
 #pragma once
 #include "common.cuh"
 #include "row_pass.cuh"
+#include "table.cuh"
 
 namespace stand {
 
@@ -47,6 +51,8 @@ struct VerifyParams {
   int* rec_ids;            // [B, D+1, K]
   float* rec_p;            // [B, D+1, K]
   unsigned long long* stats;
+  int fuse_locate;         // != 0: also run stage 1 of the N-gram update for this sequence's records
+  UpdateParams upd;        // used when fuse_locate is set
 };
 
 // Exclusive block scan of one double per thread (256 threads); returns the
@@ -73,10 +79,60 @@ __device__ __forceinline__ double block_scan_excl(double v, double* s_warp, doub
   return base + inc - v;
 }
 
+constexpr int BLOCK_CANDS = 1024;  // block-wide candidate buffer of the top-k selection
+
+// Pushes the entries of chunk `ch` of a row that reach `floor` into buf (capacity cap; *cnt keeps
+// counting past it, which the caller reads as overflow).  Called by all lanes of a warp.
+__device__ __forceinline__ void push_chunk_candidates(const void* logits, int dtype, long long row, int V, int ch,
+                                                      float floor, bool wide, uint2* buf, int* cnt, int cap, int lane) {
+#pragma unroll
+  for (int step = 0; step < 4; ++step) {
+    float f[8];
+    int idx[8];
+    if (wide && dtype == 1) {
+      const int i0 = ch * CHUNK + step * 256 + lane * 8;
+      uint4 d = make_uint4(0xFF80FF80u, 0xFF80FF80u, 0xFF80FF80u, 0xFF80FF80u);
+      if (i0 < V) d = __ldg(reinterpret_cast<const uint4*>((const unsigned short*)logits + row * (long long)V + i0));
+      ElemTraits<1>::unpack(d, f);
+#pragma unroll
+      for (int e = 0; e < 8; ++e) idx[e] = i0 + e;
+    } else if (wide) {
+      const int i0 = ch * CHUNK + step * 256 + lane * 8;
+#pragma unroll
+      for (int h = 0; h < 2; ++h) {
+        uint4 d = make_uint4(0xFF800000u, 0xFF800000u, 0xFF800000u, 0xFF800000u);
+        if (i0 + 4 * h < V) d = __ldg(reinterpret_cast<const uint4*>((const float*)logits + row * (long long)V + i0 + 4 * h));
+        f[4 * h] = __uint_as_float(d.x); f[4 * h + 1] = __uint_as_float(d.y);
+        f[4 * h + 2] = __uint_as_float(d.z); f[4 * h + 3] = __uint_as_float(d.w);
+      }
+#pragma unroll
+      for (int e = 0; e < 8; ++e) idx[e] = i0 + e;
+    } else {
+#pragma unroll
+      for (int e = 0; e < 8; ++e) {
+        idx[e] = ch * CHUNK + step * 256 + e * 32 + lane;
+        f[e] = idx[e] < V ? load_logit(logits, dtype, row * (long long)V + idx[e]) : -INFINITY;
+      }
+    }
+#pragma unroll
+    for (int e = 0; e < 8; ++e) {
+      if (f[e] >= floor && idx[e] < V) {
+        const int pos = atomicAdd(cnt, 1);
+        const float canon = f[e] == 0.0f ? 0.0f : f[e];  // -0 and +0 are one value
+        if (pos < cap) buf[pos] = make_uint2(__float_as_uint(canon), (uint32_t)idx[e]);
+      }
+    }
+  }
+}
+
 __global__ void __launch_bounds__(K2_THREADS) verify_kernel(const VerifyParams p) {
   __shared__ float s_off[NODES_MAX];
   __shared__ double s_Z[NODES_MAX];
   __shared__ double s_p[NODES_MAX][KMAX];  // target probability of candidate i of node u
+  __shared__ int s_tree[NODES_MAX], s_cn[NODES_MAX], s_fc[NODES_MAX], s_nch[NODES_MAX];
+  __shared__ int s_cid[NODES_MAX][KMAX];
+  __shared__ float s_cphi[NODES_MAX][KMAX];
+  __shared__ int s_tail[ORDER_MAX];
   __shared__ double s_scan[K2_THREADS / 32];
   __shared__ int s_path[DEPTH_MAX + 1];
   __shared__ int s_emit[DEPTH_MAX + 1];
@@ -88,23 +144,40 @@ __global__ void __launch_bounds__(K2_THREADS) verify_kernel(const VerifyParams p
   __shared__ double s_scale;         // residual target off the candidates = scale * target
   __shared__ int s_pick, s_pick_last;
   __shared__ double s_base;
-  __shared__ uint2 s_buf[K2_THREADS / 32][CAND_CAP];  // per-warp candidate buffers of the top-k selection
-  __shared__ int s_cnt[K2_THREADS / 32];
+  // top-k selection of one path row at a time
+  __shared__ float s_cmax[VOCAB_MAX / CHUNK];
+  __shared__ unsigned short s_qlist[VOCAB_MAX / CHUNK];
+  __shared__ uint2 s_cand[BLOCK_CANDS];
+  __shared__ int s_ncand, s_nq;
+  __shared__ float s_floor;
 
   const int b = blockIdx.x;
   const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
   const int N = p.N, K = p.K;
   const double cd = (double)p.c;
 
+  // ---- phase 0: stage the sequence's state ------------------------------------------
+  for (int u = tid; u < N; u += K2_THREADS) {
+    s_tree[u] = p.tree[(long long)b * N + u];
+    s_cn[u] = p.cand_n[(long long)b * N + u];
+    s_fc[u] = p.first_child[u];
+    s_nch[u] = p.n_children[u];
+  }
+  for (int i = tid; i < N * K; i += K2_THREADS) {
+    const int u = i / K, t = i - u * K;
+    s_cid[u][t] = p.cand_id[(long long)b * N * K + i];
+    s_cphi[u][t] = p.cand_phi[(long long)b * N * K + i];
+  }
+  if (tid < p.n_max) s_tail[tid] = p.tail[b * p.n_max + tid];
+  __syncthreads();
+
   // ---- phase 1 -----------------------------------------------------------
   for (int u = warp; u < N; u += K2_THREADS / 32) {
     const long long row = (long long)b * N + u;
     const RowNorm nm = row_normaliser(p.pairs + row * p.n_chunks, p.n_chunks, p.c, lane);
     if (lane == 0) { s_off[u] = nm.off; s_Z[u] = nm.Z; }
-    const int nc = p.cand_n[row];
-    if (lane < nc) {
-      const int id = p.cand_id[row * K + lane];
-      const float x = load_logit(p.logits, p.dtype, row * (long long)p.V + id);
+    if (lane < s_cn[u]) {
+      const float x = load_logit(p.logits, p.dtype, row * (long long)p.V + s_cid[u][lane]);
       s_p[u][lane] = exp2((double)x * cd - (double)nm.off) / nm.Z;
     }
   }
@@ -117,27 +190,26 @@ __global__ void __launch_bounds__(K2_THREADS) verify_kernel(const VerifyParams p
     int nsup = 0;
     double scale = 1.0;
     for (;;) {
-      const long long row = (long long)b * N + u;
-      const int fc = p.first_child[u], nch = p.n_children[u];
+      const int fc = s_fc[u], nch = s_nch[u];
       int drafted = 0;
-      while (drafted < nch && p.tree[(long long)b * N + fc + drafted] >= 0) ++drafted;
+      while (drafted < nch && s_tree[fc + drafted] >= 0) ++drafted;
       nsup = 0;
       scale = 1.0;
       if (drafted == 0) break;  // nothing drafted below u: sample from its target
-      const int nc = p.cand_n[row];
+      const int nc = s_cn[u];
       double q[KMAX], pt[KMAX];
       int cid[KMAX];
       double phis = 0.0;
       for (int i = 0; i < nc; ++i) {
-        cid[i] = p.cand_id[row * K + i];
-        q[i] = (double)p.cand_phi[row * K + i];
+        cid[i] = s_cid[u][i];
+        q[i] = (double)s_cphi[u][i];
         phis += q[i];
         pt[i] = s_p[u][i];
       }
       for (int i = 0; i < nc; ++i) q[i] /= phis;
       int accepted = -1;
       for (int j = 0; j < drafted; ++j) {
-        const int x = p.tree[(long long)b * N + fc + j];
+        const int x = s_tree[fc + j];
         int ix = -1;
         for (int i = 0; i < nc; ++i)
           if (cid[i] == x) ix = i;
@@ -156,7 +228,7 @@ __global__ void __launch_bounds__(K2_THREADS) verify_kernel(const VerifyParams p
           for (int i = 0; i < nc; ++i) q[i] /= qs;
       }
       if (accepted >= 0) {
-        s_emit[m] = p.tree[(long long)b * N + fc + accepted];
+        s_emit[m] = s_tree[fc + accepted];
         u = fc + accepted;
         ++m;
         s_path[m] = u;
@@ -277,7 +349,7 @@ __global__ void __launch_bounds__(K2_THREADS) verify_kernel(const VerifyParams p
     s_emit[m] = y;
     // context windows of the accepted rows, then the advanced tail
     int win[ORDER_MAX];
-    for (int i = 0; i < p.n_max; ++i) win[i] = p.tail[b * p.n_max + i];
+    for (int i = 0; i < p.n_max; ++i) win[i] = s_tail[i];
     for (int j = 0; j <= m; ++j) {
       for (int i = 0; i < p.n_max; ++i) p.rec_ctx[((long long)b * W1 + j) * p.n_max + i] = win[i];
       for (int i = 0; i + 1 < p.n_max; ++i) win[i] = win[i + 1];
@@ -297,26 +369,78 @@ __global__ void __launch_bounds__(K2_THREADS) verify_kernel(const VerifyParams p
     if (p.emitted_user) p.emitted_user[b * W1 + tid] = e;
     p.path[b * W1 + tid] = tid <= m ? s_path[tid] : -1;
   }
-  // compressed rows of the accepted path: the exact top-k of each row, as probabilities
-  for (int j = warp; j <= m; j += K2_THREADS / 32) {
+  // Compressed rows of the accepted path: the exact top-k of each row, as probabilities.  The k-th
+  // largest chunk maximum bounds the k-th largest entry from below, so only the chunks whose maximum
+  // reaches it (about k) are read again, one chunk per warp.
+  const bool wide = p.dtype == 1 ? (((uintptr_t)p.logits & 15) == 0 && (p.V & 7) == 0)
+                                 : (((uintptr_t)p.logits & 15) == 0 && (p.V & 3) == 0);
+  for (int j = 0; j <= m; ++j) {
     const int u = s_path[j];
     const long long row = (long long)b * N + u;
-    const float o = s_off[u];
-    const double z = s_Z[u];
-    const int n = row_topk_warp(p.logits, p.dtype, row, p.V, p.pairs + row * p.n_chunks, p.n_chunks, K, s_buf[warp],
-                                &s_cnt[warp], lane);
-    if (lane < K) {
-      const long long at = ((long long)b * W1 + j) * K + lane;
-      if (lane < n) {
-        const uint2 e = s_buf[warp][lane];
-        p.rec_ids[at] = (int)e.y;
-        p.rec_p[at] = (float)(exp2((double)__uint_as_float(e.x) * cd - (double)o) / z);
+    const float2* pairs = p.pairs + row * p.n_chunks;
+    for (int ch = tid; ch < p.n_chunks; ch += K2_THREADS) s_cmax[ch] = pairs[ch].y;
+    if (tid == 0) { s_ncand = 0; s_nq = 0; }
+    __syncthreads();
+    if (warp == 0) {
+      float tau = -INFINITY;
+      if (p.n_chunks >= K) {
+        unsigned long long below = ~0ull;
+        for (int r = 0; r < K; ++r) {
+          unsigned long long best = 0ull;
+          for (int ch = lane; ch < p.n_chunks; ch += 32) {
+            const unsigned long long key = select_key(__float_as_uint(s_cmax[ch]), (uint32_t)ch);
+            if (key < below && key > best) best = key;
+          }
+          below = warp_max_u64(best);
+        }
+        tau = key_value(below);
+      }
+      if (lane == 0) s_floor = tau;
+    }
+    __syncthreads();
+    const float floor = s_floor;
+    for (int ch = tid; ch < p.n_chunks; ch += K2_THREADS)
+      if (s_cmax[ch] >= floor) s_qlist[atomicAdd(&s_nq, 1)] = (unsigned short)ch;
+    __syncthreads();
+    const int nq = s_nq;
+    for (int qi = warp; qi < nq; qi += K2_THREADS / 32)
+      push_chunk_candidates(p.logits, p.dtype, row, p.V, (int)s_qlist[qi], floor, wide, s_cand, &s_ncand, BLOCK_CANDS, lane);
+    __syncthreads();
+    if (warp == 0) {
+      int n = s_ncand;
+      if (n > BLOCK_CANDS) {
+        // more entries reach the bound than the buffer holds (long runs of equal values): the streaming
+        // selection copes with any input, one chunk at a time
+        n = row_topk_warp(p.logits, p.dtype, row, p.V, pairs, p.n_chunks, K, s_cand, &s_ncand, lane);
       } else {
-        p.rec_ids[at] = -1;
-        p.rec_p[at] = 0.0f;
+        if (n > 0) compact_topk(s_cand, &s_ncand, n, K, lane, floor);
+        n = n < K ? n : K;
+      }
+      if (lane < K) {
+        const long long at = ((long long)b * W1 + j) * K + lane;
+        if (lane < n) {
+          const uint2 e = s_cand[lane];
+          p.rec_ids[at] = (int)e.y;
+          p.rec_p[at] = (float)(exp2((double)__uint_as_float(e.x) * cd - (double)s_off[u]) / s_Z[u]);
+        } else {
+          p.rec_ids[at] = -1;
+          p.rec_p[at] = 0.0f;
+        }
       }
     }
-    __syncwarp();
+    __syncthreads();
+  }
+
+  // ---- stage 1 of the table update for this sequence's records (8 lanes per record) -----
+  if (p.fuse_locate) {
+    const int n_rec = W1 * p.n_max;
+    for (int r0 = 0; r0 < n_rec; r0 += K2_THREADS / GROUP) {
+      const int r = r0 + tid / GROUP;
+      const bool in_range = r < n_rec;
+      const int j = in_range ? r / p.n_max : 0;
+      const int n = in_range ? r - j * p.n_max + 1 : 1;
+      locate_record(p.upd, (long long)b * W1 + j, n, in_range);
+    }
   }
 }
 
