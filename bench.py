@@ -202,6 +202,19 @@ def run_ours(args, rank, world, local):
     gpu.profile_row_pass(None, None)
     torch.cuda.synchronize()
     k1_ms = statistics.mean(a.elapsed_time(b) for a, b in evs)
+    # the same steps with events at every stage boundary (diagnostic: where the rest of a step goes)
+    n_st = min(args.steps, 100)
+    sev = [[torch.cuda.Event(enable_timing=True) for _ in range(5)] for _ in range(n_st)]
+    for row in sev:
+        for e in row:
+            e.record()
+    for s in range(n_st):
+        gpu.profile_stages(sev[s])
+        gpu.step(ring[s % ring_n])
+    gpu.profile_stages(None)
+    torch.cuda.synchronize()
+    stage_us = {name: 1e3 * statistics.mean(row[i].elapsed_time(row[i + 1]) for row in sev)
+                for i, name in enumerate(("row_pass", "verify", "update", "draft"))}
     clocks = sampler.stop()
 
     if dist is not None:
@@ -261,6 +274,7 @@ def run_ours(args, rank, world, local):
                        if world > 1 else "single GPU", "acceptance_length": accept_len},
             "clocks": clocks, "e2e": e2e, "gpu_launches": int(launches), "roofline": roofline,
             "logits_gbs": alg_bytes * world / (ms_per_step * 1e-3) / 1e9,
+            "stage_us": stage_us,
             "table": {"drops": st["drops"], "max_probe": st["max_probe_seen"], "lookup_hits": st["lookup_hits"],
                       "lookups": st["lookups"]},
         }

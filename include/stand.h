@@ -223,6 +223,11 @@ int stand_state_load(stand_ctx* ctx, const int32_t* dev_tail, const int64_t* dev
  * after it, so the caller can time that kernel alone.  NULL, NULL switches the hook off. */
 int stand_profile_row_pass(stand_ctx* ctx, void* ev_before, void* ev_after);
 
+/* Timing hook for benchmarks: events [5] (cudaEvent_t as void*, any may be NULL) are recorded on the
+ * stream by every later step at: before the row pass, after it, after the verification walk, after the
+ * table update, after drafting.  A NULL array switches the hook off. */
+int stand_profile_stages(stand_ctx* ctx, void* const* events);
+
 /* How many kernels the library has launched through this context so far. */
 uint64_t stand_launch_count(const stand_ctx* ctx);
 

@@ -20,7 +20,7 @@ EXPORTS = [
     "stand_ngram_update", "stand_ngram_update_bulk", "stand_draft_tree", "stand_step", "stand_step_host",
     "stand_row_stats_scratch_bytes", "stand_row_stats", "stand_row_stats_static", "stand_get_stats",
     "stand_last_path", "stand_tree_depth", "stand_table_dump", "stand_table_load", "stand_state_dump",
-    "stand_state_load", "stand_profile_row_pass", "stand_launch_count", "stand_strerror",
+    "stand_state_load", "stand_profile_row_pass", "stand_profile_stages", "stand_launch_count", "stand_strerror",
 ]
 
 
@@ -84,6 +84,8 @@ def lib():
     L.stand_state_load.argtypes = [vp, vp, vp, vp, vp, vp, vp, u32, vp]
     L.stand_profile_row_pass.argtypes = [vp, vp, vp]
     L.stand_profile_row_pass.restype = C.c_int
+    L.stand_profile_stages.argtypes = [vp, C.POINTER(vp)]
+    L.stand_profile_stages.restype = C.c_int
     L.stand_launch_count.argtypes = [vp]
     L.stand_launch_count.restype = u64
     L.stand_strerror.argtypes = [C.c_int]
@@ -233,6 +235,15 @@ class Stand:
         a = None if ev_before is None else C.c_void_p(ev_before.cuda_event)
         b = None if ev_after is None else C.c_void_p(ev_after.cuda_event)
         _check(lib().stand_profile_row_pass(self.h, a, b), "stand_profile_row_pass")
+
+    def profile_stages(self, events=None):
+        """Five torch.cuda.Event (already recorded once, enable_timing=True) recorded at the stage boundaries of
+        every later step: before/after the row pass, after verification, after the update, after drafting."""
+        if events is None:
+            _check(lib().stand_profile_stages(self.h, None), "stand_profile_stages")
+            return
+        arr = (C.c_void_p * 5)(*[C.c_void_p(e.cuda_event) for e in events])
+        _check(lib().stand_profile_stages(self.h, arr), "stand_profile_stages")
 
     def lens_device(self, out):
         """Copies the sequence lengths into `out` (int64 [B], device) on the current stream."""

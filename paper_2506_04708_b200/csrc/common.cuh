@@ -62,13 +62,48 @@ __device__ __forceinline__ double warp_sum_d(double v) {
   for (int o = 16; o > 0; o >>= 1) v += __shfl_xor_sync(FULL, v, o);
   return v;
 }
+__device__ __forceinline__ uint32_t warp_max_u32(uint32_t v) {
+  uint32_t m;
+  asm volatile("redux.sync.max.u32 %0, %1, 0xffffffff;" : "=r"(m) : "r"(v));
+  return m;
+}
+// 64-bit maximum as two passes through the integer reduction unit: high words, then the low words of
+// the lanes that hold the largest high word.
 __device__ __forceinline__ unsigned long long warp_max_u64(unsigned long long v) {
-#pragma unroll
-  for (int o = 16; o > 0; o >>= 1) {
-    const unsigned long long w = __shfl_xor_sync(FULL, v, o);
-    v = w > v ? w : v;
-  }
-  return v;
+  const uint32_t hi = (uint32_t)(v >> 32), lo = (uint32_t)v;
+  const uint32_t mh = warp_max_u32(hi);
+  const uint32_t ml = warp_max_u32(hi == mh ? lo : 0u);
+  return ((unsigned long long)mh << 32) | ml;
+}
+
+// ---------------------------------------------------------------------------
+// Short double-precision helpers for the serial parts of the step (a library exp2 or scalbn costs
+// several times as many dependent instructions).
+// ---------------------------------------------------------------------------
+// 2^k exactly; 0 below the normal range (such terms are far below one ulp of any sum they enter).
+__device__ __forceinline__ double pow2_int(int k) {
+  if (k < -1022) return 0.0;
+  if (k > 1023) k = 1023;
+  return __longlong_as_double((long long)(k + 1023) << 52);
+}
+// 2^t for t <= ~1000, relative error below 1e-14: t = n + f, |f| <= 1/2, Taylor series of 2^f to degree 11.
+__device__ __forceinline__ double exp2_d(double t) {
+  if (!(t > -1100.0)) return 0.0;
+  const int n = __double2int_rn(t);
+  const double f = (t - (double)n) * 0.6931471805599453094;
+  double r = 1.0 / 39916800.0;
+  r = fma(r, f, 1.0 / 3628800.0);
+  r = fma(r, f, 1.0 / 362880.0);
+  r = fma(r, f, 1.0 / 40320.0);
+  r = fma(r, f, 1.0 / 5040.0);
+  r = fma(r, f, 1.0 / 720.0);
+  r = fma(r, f, 1.0 / 120.0);
+  r = fma(r, f, 1.0 / 24.0);
+  r = fma(r, f, 1.0 / 6.0);
+  r = fma(r, f, 0.5);
+  r = fma(r, f, 1.0);
+  r = fma(r, f, 1.0);
+  return r * pow2_int(n);
 }
 
 // Order-preserving map float bits -> uint32 (larger float = larger integer).

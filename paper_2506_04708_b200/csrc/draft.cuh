@@ -35,9 +35,28 @@ struct DraftParams {
   unsigned long long* stats;
 };
 
+// Rank of this lane's candidate by g = log(phi) - log(-log U) in double precision (larger first, equal
+// scores by lower id).  Called by all lanes of a warp; kept out of line: it runs for about one node in a hundred.
+__device__ __noinline__ int gumbel_rank_double(bool valid, int id, float phi, uint32_t u24) {
+  double g = 0.0;
+  if (valid) {
+    const double U = ((double)u24 + 0.5) * (1.0 / 16777216.0);
+    g = log((double)phi) - log(-log(U));
+  }
+  int rank = 0;
+  for (int j = 0; j < KMAX; ++j) {
+    const double gj = __shfl_sync(FULL, g, j);
+    const int idj = __shfl_sync(FULL, id, j);
+    const bool vj = __shfl_sync(FULL, (int)valid, j) != 0;
+    if (vj && (gj > g || (gj == g && idj < id))) ++rank;
+  }
+  return rank;
+}
+
 __global__ void __launch_bounds__(K4_THREADS) draft_kernel(const DraftParams p) {
   __shared__ int s_tok[NODES_MAX], s_parent[NODES_MAX], s_fc[NODES_MAX], s_nch[NODES_MAX];
   __shared__ int s_tail[ORDER_MAX], s_level[DEPTH_MAX + 2];
+  __shared__ Slot s_slot[K4_THREADS / 32];  // per warp: the slot that won the lookup
   const int b = blockIdx.x, tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
   const int N = p.N, K = p.K, n_max = p.n_max;
   // topology and tail once, with coalesced loads: the level loop below touches shared memory only
@@ -80,7 +99,9 @@ __global__ void __launch_bounds__(K4_THREADS) draft_kernel(const DraftParams p) 
           key[4 - n + i] = t;
         }
       }
-      uint32_t slot = find_slot_group(p.table, p.mask, p.max_probe, key, ok);
+      uint4 line[8];
+      int src_lane;
+      uint32_t slot = find_slot_group_fetch(p.table, p.mask, p.max_probe, key, ok, line, &src_lane);
       const unsigned found = __ballot_sync(FULL, slot != NO_SLOT);
       unsigned hits = 0;  // bit n-1: order n matched
       for (int gq = 0; gq < 32 / GROUP; ++gq)
@@ -91,25 +112,42 @@ __global__ void __launch_bounds__(K4_THREADS) draft_kernel(const DraftParams p) 
       }
       if (hits == 0) { if (lane == 0) p.cand_n[row] = 0; continue; }
       const int winner = 31 - __clz(hits);  // the longest order that matched
-      slot = __shfl_sync(FULL, slot, winner * GROUP);
-      const Slot* s = &p.table[slot];
+      // the lane that probed the winning slot already holds its contents: hand them to the warp
+      src_lane = __shfl_sync(FULL, src_lane, winner * GROUP);
+      uint4* img = reinterpret_cast<uint4*>(&s_slot[warp]);
+      if (lane == src_lane) {
+#pragma unroll
+        for (int t = 0; t < 8; ++t) img[t] = line[t];
+      }
+      __syncwarp();
+      const Slot* s = &s_slot[warp];
       const int n_items = (int)s->n_items;
       int id = -1;
       float phi = 0.0f;
       if (lane < n_items && lane < K) { id = s->ids[lane]; phi = s->probs[lane]; }
+      __syncwarp();
       const bool valid = id >= 0 && phi > 0.0f;
-      double g = 0.0;
+      // Perturbed scores in single precision first; they decide the order whenever every pair of
+      // candidates is further apart than single precision can blur (1e-3 against errors of a few 1e-6).
+      // Otherwise the scores are formed again in double precision.
+      const uint32_t u24 = valid ? philox_u24(p.seed, b, p.step, u, SLOT_GUMBEL | (uint32_t)id) : 0u;
+      float gf = 0.0f;
       if (valid) {
-        const double U = ((double)philox_u24(p.seed, b, p.step, u, SLOT_GUMBEL | (uint32_t)id) + 0.5) * (1.0 / 16777216.0);
-        g = log((double)phi) - log(-log(U));
+        // -log U with U = (u24 + 1/2) / 2^24: above one half through log1p of the exact complement
+        const float L = u24 < (1u << 23) ? -logf(((float)u24 + 0.5f) * (1.0f / 16777216.0f))
+                                         : -log1pf(-((float)(16777216u - u24) - 0.5f) * (1.0f / 16777216.0f));
+        gf = logf(phi) - logf(L);
       }
       int rank = 0;
+      bool close = false;
       for (int j = 0; j < KMAX; ++j) {
-        const double gj = __shfl_sync(FULL, g, j);
+        const float gj = __shfl_sync(FULL, gf, j);
         const int idj = __shfl_sync(FULL, id, j);
         const bool vj = __shfl_sync(FULL, (int)valid, j) != 0;
-        if (vj && (gj > g || (gj == g && idj < id))) ++rank;
+        if (vj && (gj > gf || (gj == gf && idj < id))) ++rank;
+        if (vj && j != lane && fabsf(gj - gf) < 1e-3f) close = true;
       }
+      if (__any_sync(FULL, valid && close)) rank = gumbel_rank_double(valid, id, phi, u24);
       if (valid && rank < m) s_tok[s_fc[u] + rank] = id;
       const unsigned vmask = __ballot_sync(FULL, valid);
       if (valid) {

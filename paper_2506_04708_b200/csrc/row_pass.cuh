@@ -360,7 +360,7 @@ __device__ __forceinline__ RowNorm row_normaliser(const float2* pairs, int n_chu
   double z = 0.0;
   for (int ch = lane; ch < n_chunks; ch += 32) {
     const float2 pr = pairs[ch];
-    if (pr.x > 0.0f) z += scalbn((double)pr.x, (int)(chunk_offset(pr.y, c) - om));
+    if (pr.x > 0.0f) z += (double)pr.x * pow2_int((int)(chunk_offset(pr.y, c) - om));
   }
   RowNorm r;
   r.off = om;
@@ -370,7 +370,7 @@ __device__ __forceinline__ RowNorm row_normaliser(const float2* pairs, int n_chu
 
 // Mass of one chunk relative to the row offset `off` (before division by Z).
 __device__ __forceinline__ double chunk_mass(float2 pr, float c, float off) {
-  return pr.x > 0.0f ? scalbn((double)pr.x, (int)(chunk_offset(pr.y, c) - off)) : 0.0;
+  return pr.x > 0.0f ? (double)pr.x * pow2_int((int)(chunk_offset(pr.y, c) - off)) : 0.0;
 }
 
 // Keeps the k best of the n buffered candidates at buf[0..k), best first; returns
@@ -529,7 +529,7 @@ __global__ void __launch_bounds__(FIN_WARPS * 32) row_finalize_kernel(const RowF
       const float x = __uint_as_float(e.x);
       p.ids[at] = (int)e.y;
       p.values[at] = x;
-      p.probs[at] = (float)(exp2((double)x * (double)p.c - (double)nm.off) / nm.Z);
+      p.probs[at] = (float)(exp2_d((double)x * (double)p.c - (double)nm.off) / nm.Z);
     } else {
       p.ids[at] = -1;
       p.values[at] = 0.0f;

@@ -110,6 +110,7 @@ struct stand_ctx {
   int max_probe;
   float c;  // log2(e) / T
   cudaEvent_t ev_before, ev_after;  // optional timing hook around the row pass
+  cudaEvent_t ev_stage[5];          // optional timing hook at the stage boundaries of a step
 
   template <typename T> T* at(size_t off) const { return reinterpret_cast<T*>(ws + off); }
   int* topo_parent() const { return at<int>(L.topo); }
@@ -202,10 +203,12 @@ UpdateParams step_update_params(stand_ctx* x) {
 int run_verify(stand_ctx* x, const void* logits, int32_t* emitted, int32_t* n_emitted, bool fuse_locate, cudaStream_t st) {
   const stand_config& c = x->cfg;
   if (x->ev_before) cudaEventRecord(x->ev_before, st);
+  if (x->ev_stage[0]) cudaEventRecord(x->ev_stage[0], st);
   int rc = launch_row_pass(logits, (long long)c.B * c.N, c.V, c.dtype, x->d.n_chunks, x->c, x->at<float2>(x->L.pairs),
                            x->at<int>(x->L.status), st);
   if (rc) return rc;
   if (x->ev_after) cudaEventRecord(x->ev_after, st);
+  if (x->ev_stage[1]) cudaEventRecord(x->ev_stage[1], st);
   x->launches += 1;
   x->step += 1;  // the tree drafted in step s-1 is verified in step s
   VerifyParams v;
@@ -224,6 +227,7 @@ int run_verify(stand_ctx* x, const void* logits, int32_t* emitted, int32_t* n_em
   verify_kernel<<<c.B, K2_THREADS, 0, st>>>(v);
   rc = launch_ok();
   if (rc) return rc;
+  if (x->ev_stage[2]) cudaEventRecord(x->ev_stage[2], st);
   x->launches += 1;
   x->pending = true;
   x->located = fuse_locate;
@@ -249,6 +253,7 @@ int run_update_rows(stand_ctx* x, const UpdateParams& u, bool located, cudaStrea
 int run_update(stand_ctx* x, cudaStream_t st) {
   const int rc = run_update_rows(x, step_update_params(x), x->located, st);
   if (rc == STAND_OK) { x->pending = false; x->located = false; }
+  if (x->ev_stage[3]) cudaEventRecord(x->ev_stage[3], st);
   return rc;
 }
 
@@ -264,6 +269,7 @@ int run_draft(stand_ctx* x, int32_t* tree_user, cudaStream_t st) {
   draft_kernel<<<c.B, K4_THREADS, 0, st>>>(d);
   const int rc = launch_ok();
   if (rc == STAND_OK) x->launches += 1;
+  if (x->ev_stage[4]) cudaEventRecord(x->ev_stage[4], st);
   return rc;
 }
 
@@ -310,6 +316,7 @@ int stand_init(const stand_config* cfg, void* dev_workspace, size_t bytes, stand
   x->max_probe = cfg->max_probe > 0 ? cfg->max_probe : 96;
   x->ev_before = nullptr;
   x->ev_after = nullptr;
+  for (int i = 0; i < 5; ++i) x->ev_stage[i] = nullptr;
   x->c = log2e_over_T(cfg->temperature);
 
   int topo[4 * NODES_MAX + DEPTH_MAX + 2];
@@ -615,6 +622,12 @@ int stand_profile_row_pass(stand_ctx* x, void* ev_before, void* ev_after) {
   if (!x || ((ev_before == nullptr) != (ev_after == nullptr))) return STAND_E_ARG;
   x->ev_before = (cudaEvent_t)ev_before;
   x->ev_after = (cudaEvent_t)ev_after;
+  return STAND_OK;
+}
+
+int stand_profile_stages(stand_ctx* x, void* const* events) {
+  if (!x) return STAND_E_ARG;
+  for (int i = 0; i < 5; ++i) x->ev_stage[i] = events ? (cudaEvent_t)events[i] : nullptr;
   return STAND_OK;
 }
 

@@ -182,6 +182,43 @@ __device__ __forceinline__ uint32_t find_slot_group(const Slot* table, unsigned 
   return result;
 }
 
+// Read-only lookup that also brings the whole 128-byte slot: every probing lane reads its slot's eight
+// 16-byte words at once, so a hit costs one memory round trip instead of two (key, then contents).
+// Returns the slot index or NO_SLOT; *src_lane is the lane that holds the matching slot in `line`.
+// Called by ALL 32 lanes of a warp, 8 lanes per key.
+__device__ __forceinline__ uint32_t find_slot_group_fetch(const Slot* table, unsigned long long mask, int max_probe,
+                                                          const int (&key)[4], bool live, uint4 (&line)[8], int* src_lane) {
+  const int lane = threadIdx.x & 31, gl = lane & (GROUP - 1), gbase = lane & ~(GROUP - 1);
+  const ProbeSeq ps = probe_seq(key, mask);
+  uint32_t result = NO_SLOT;
+  *src_lane = gbase;
+  bool done = !live;
+  for (int base = 0; __any_sync(FULL, !done); base += GROUP) {
+    if (base >= max_probe) done = true;
+    const int i = base + gl;
+    const unsigned long long s = (ps.start + (unsigned long long)i * ps.stride) & mask;
+    int st = 0;
+    if (!done && i < max_probe) {
+      const uint4* w = reinterpret_cast<const uint4*>(&table[s]);
+#pragma unroll
+      for (int t = 0; t < 8; ++t) line[t] = w[t];
+      const uint4 k = line[0];
+      st = ((int)k.x == key[0] && (int)k.y == key[1] && (int)k.z == key[2] && (int)k.w == key[3]) ? 1
+           : ((k.x & k.y & k.z & k.w) == 0xFFFFFFFFu ? 2 : 0);
+    }
+    const unsigned votes = __ballot_sync(FULL, !done && st != 0);
+    const unsigned mine_votes = (votes >> gbase) & ((1u << GROUP) - 1u);
+    const int first = mine_votes ? __ffs(mine_votes) - 1 : 0;
+    const int st_first = __shfl_sync(FULL, st, gbase + first);
+    const unsigned long long s_first = __shfl_sync(FULL, s, gbase + first);
+    if (!done && mine_votes != 0) {
+      if (st_first == 1) { result = (uint32_t)s_first; *src_lane = gbase + first; }
+      done = true;  // the key, or a free position before it: absent
+    }
+  }
+  return result;
+}
+
 __global__ void table_clear_kernel(Slot* table, unsigned long long n_slots) {
   // one thread per 16 bytes: 8 per slot
   const unsigned long long i = (unsigned long long)blockIdx.x * blockDim.x + threadIdx.x;

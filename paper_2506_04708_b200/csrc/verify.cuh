@@ -4,8 +4,8 @@
 //   phase 0 (all warps)  the sequence's tree, candidate lists and topology are staged in
 //                        shared memory with one round of coalesced loads;
 //   phase 1 (all warps)  normaliser of every row of the sequence from the chunk
-//                        pairs, and the target probability of every drafted
-//                        candidate (a handful of gathered logits per node);
+//                        pairs (8 lanes per row), and the target probability of every
+//                        drafted candidate (one round of gathered logits);
 //   phase 2 (thread 0)   the walk: children in draft order, accept iff
 //                        U * q(x) < p~(x); on rejection p~ <- norm(max(0, p~ - q)),
 //                        x leaves q; off the candidate list p~ is the target scaled
@@ -79,7 +79,9 @@ __device__ __forceinline__ double block_scan_excl(double v, double* s_warp, doub
   return base + inc - v;
 }
 
-constexpr int BLOCK_CANDS = 1024;  // block-wide candidate buffer of the top-k selection
+constexpr int TOPK_ROWS = 4;       // path rows whose top-k is selected together
+constexpr int TOPK_ITEMS = 1024;   // (row, chunk) work items per group of rows
+constexpr int ROW_LANES = 8;       // lanes that share one row in the normaliser phase
 
 // Pushes the entries of chunk `ch` of a row that reach `floor` into buf (capacity cap; *cnt keeps
 // counting past it, which the caller reads as overflow).  Called by all lanes of a warp.
@@ -144,12 +146,12 @@ __global__ void __launch_bounds__(K2_THREADS) verify_kernel(const VerifyParams p
   __shared__ double s_scale;         // residual target off the candidates = scale * target
   __shared__ int s_pick, s_pick_last;
   __shared__ double s_base;
-  // top-k selection of one path row at a time
-  __shared__ float s_cmax[VOCAB_MAX / CHUNK];
-  __shared__ unsigned short s_qlist[VOCAB_MAX / CHUNK];
-  __shared__ uint2 s_cand[BLOCK_CANDS];
-  __shared__ int s_ncand, s_nq;
-  __shared__ float s_floor;
+  __shared__ double s_q[KMAX], s_pt[KMAX];  // the walk's draft and residual target distributions
+  // top-k selection of up to TOPK_ROWS path rows at a time
+  __shared__ uint32_t s_items[TOPK_ITEMS];  // (row slot << 16) | chunk: chunks that can hold a top-k entry
+  __shared__ uint2 s_cand[TOPK_ROWS][CAND_CAP];
+  __shared__ int s_ncand[TOPK_ROWS], s_nitems;
+  __shared__ float s_floor[TOPK_ROWS];
 
   const int b = blockIdx.x;
   const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
@@ -171,14 +173,35 @@ __global__ void __launch_bounds__(K2_THREADS) verify_kernel(const VerifyParams p
   if (tid < p.n_max) s_tail[tid] = p.tail[b * p.n_max + tid];
   __syncthreads();
 
-  // ---- phase 1 -----------------------------------------------------------
-  for (int u = warp; u < N; u += K2_THREADS / 32) {
-    const long long row = (long long)b * N + u;
-    const RowNorm nm = row_normaliser(p.pairs + row * p.n_chunks, p.n_chunks, p.c, lane);
-    if (lane == 0) { s_off[u] = nm.off; s_Z[u] = nm.Z; }
-    if (lane < s_cn[u]) {
-      const float x = load_logit(p.logits, p.dtype, row * (long long)p.V + s_cid[u][lane]);
-      s_p[u][lane] = exp2((double)x * cd - (double)nm.off) / nm.Z;
+  // ---- phase 1: normalisers (8 lanes per row), then all candidate logits in one round of gathers ----
+  {
+    const int gl = tid & (ROW_LANES - 1);
+    for (int u0 = 0; u0 < N; u0 += K2_THREADS / ROW_LANES) {
+      const int u = u0 + tid / ROW_LANES;
+      const bool live = u < N;
+      const float2* pairs = p.pairs + ((long long)b * N + (live ? u : 0)) * p.n_chunks;
+      float om = -INFINITY;
+      if (live)
+        for (int ch = gl; ch < p.n_chunks; ch += ROW_LANES) {
+          const float2 pr = pairs[ch];
+          if (pr.x > 0.0f) om = fmaxf(om, chunk_offset(pr.y, p.c));
+        }
+#pragma unroll
+      for (int o = ROW_LANES / 2; o > 0; o >>= 1) om = fmaxf(om, __shfl_xor_sync(FULL, om, o));
+      double z = 0.0;
+      if (live)
+        for (int ch = gl; ch < p.n_chunks; ch += ROW_LANES) z += chunk_mass(pairs[ch], p.c, om);
+#pragma unroll
+      for (int o = ROW_LANES / 2; o > 0; o >>= 1) z += __shfl_xor_sync(FULL, z, o);
+      if (live && gl == 0) { s_off[u] = om; s_Z[u] = z; }
+    }
+  }
+  __syncthreads();
+  for (int i = tid; i < N * KMAX; i += K2_THREADS) {
+    const int u = i / KMAX, t = i - u * KMAX;
+    if (t < s_cn[u]) {
+      const float x = load_logit(p.logits, p.dtype, ((long long)b * N + u) * (long long)p.V + s_cid[u][t]);
+      s_p[u][t] = exp2_d((double)x * cd - (double)s_off[u]) / s_Z[u];
     }
   }
   __syncthreads();
@@ -197,35 +220,34 @@ __global__ void __launch_bounds__(K2_THREADS) verify_kernel(const VerifyParams p
       scale = 1.0;
       if (drafted == 0) break;  // nothing drafted below u: sample from its target
       const int nc = s_cn[u];
-      double q[KMAX], pt[KMAX];
-      int cid[KMAX];
       double phis = 0.0;
-      for (int i = 0; i < nc; ++i) {
-        cid[i] = s_cid[u][i];
-        q[i] = (double)s_cphi[u][i];
-        phis += q[i];
-        pt[i] = s_p[u][i];
-      }
-      for (int i = 0; i < nc; ++i) q[i] /= phis;
+      for (int i = 0; i < nc; ++i) phis += (double)s_cphi[u][i];
+      const double inv_phis = 1.0 / phis;
+      for (int i = 0; i < nc; ++i) { s_q[i] = (double)s_cphi[u][i] * inv_phis; s_pt[i] = s_p[u][i]; }
       int accepted = -1;
       for (int j = 0; j < drafted; ++j) {
         const int x = s_tree[fc + j];
         int ix = -1;
         for (int i = 0; i < nc; ++i)
-          if (cid[i] == x) ix = i;
+          if (s_cid[u][i] == x) ix = i;
         const double U = (double)philox_u24(p.seed, b, p.step, u, (uint32_t)j) * (1.0 / 16777216.0);
-        if (ix < 0 || U * q[ix] < pt[ix]) { accepted = j; break; }
+        if (ix < 0 || U * s_q[ix] < s_pt[ix]) { accepted = j; break; }
         // rejected: residual target, x leaves the draft distribution
         double overlap = 0.0;
-        for (int i = 0; i < nc; ++i) overlap += fmin(pt[i], q[i]);
-        const double zr = 1.0 - overlap;
-        for (int i = 0; i < nc; ++i) pt[i] = fmax(0.0, pt[i] - q[i]) / zr;
-        scale /= zr;
-        q[ix] = 0.0;
+        for (int i = 0; i < nc; ++i) overlap += fmin(s_pt[i], s_q[i]);
+        const double inv_zr = 1.0 / (1.0 - overlap);
         double qs = 0.0;
-        for (int i = 0; i < nc; ++i) qs += q[i];
-        if (qs > 0.0)
-          for (int i = 0; i < nc; ++i) q[i] /= qs;
+        for (int i = 0; i < nc; ++i) {
+          const double qi = s_q[i];
+          s_pt[i] = fmax(0.0, s_pt[i] - qi) * inv_zr;
+          if (i != ix) qs += qi;
+        }
+        s_q[ix] = 0.0;
+        scale *= inv_zr;
+        if (qs > 0.0) {
+          const double inv_qs = 1.0 / qs;
+          for (int i = 0; i < nc; ++i) s_q[i] *= inv_qs;
+        }
       }
       if (accepted >= 0) {
         s_emit[m] = s_tree[fc + accepted];
@@ -235,7 +257,7 @@ __global__ void __launch_bounds__(K2_THREADS) verify_kernel(const VerifyParams p
         continue;
       }
       nsup = nc;
-      for (int i = 0; i < nc; ++i) { s_sup_id[i] = cid[i]; s_sup_pt[i] = pt[i]; s_sup_p[i] = s_p[u][i]; }
+      for (int i = 0; i < nc; ++i) { s_sup_id[i] = s_cid[u][i]; s_sup_pt[i] = s_pt[i]; s_sup_p[i] = s_p[u][i]; }
       break;
     }
     s_m = m;
@@ -319,7 +341,7 @@ __global__ void __launch_bounds__(K2_THREADS) verify_kernel(const VerifyParams p
       if (s_hit >= 0) w[e] = s_sup_pt[s_hit];
       else {
         const float x = load_logit(p.logits, p.dtype, rows * (long long)p.V + v);
-        w[e] = scale * (exp2((double)x * cd - (double)off) / Z);
+        w[e] = scale * (exp2_d((double)x * cd - (double)off) / Z);
       }
     }
     wsum += w[e];
@@ -371,57 +393,67 @@ __global__ void __launch_bounds__(K2_THREADS) verify_kernel(const VerifyParams p
   }
   // Compressed rows of the accepted path: the exact top-k of each row, as probabilities.  The k-th
   // largest chunk maximum bounds the k-th largest entry from below, so only the chunks whose maximum
-  // reaches it (about k) are read again, one chunk per warp.
+  // reaches it (about k per row) are read again.  Up to TOPK_ROWS rows go through together: one warp
+  // per row finds the bound and lists the row's chunks, all warps share the chunk reads, one warp
+  // per row selects.
   const bool wide = p.dtype == 1 ? (((uintptr_t)p.logits & 15) == 0 && (p.V & 7) == 0)
                                  : (((uintptr_t)p.logits & 15) == 0 && (p.V & 3) == 0);
-  for (int j = 0; j <= m; ++j) {
-    const int u = s_path[j];
-    const long long row = (long long)b * N + u;
-    const float2* pairs = p.pairs + row * p.n_chunks;
-    for (int ch = tid; ch < p.n_chunks; ch += K2_THREADS) s_cmax[ch] = pairs[ch].y;
-    if (tid == 0) { s_ncand = 0; s_nq = 0; }
+  for (int j0 = 0; j0 <= m; j0 += TOPK_ROWS) {
+    const int nr = min(TOPK_ROWS, m + 1 - j0);
+    if (tid < TOPK_ROWS) s_ncand[tid] = 0;
+    if (tid == 0) s_nitems = 0;
     __syncthreads();
-    if (warp == 0) {
+    if (warp < nr) {
+      const float2* pairs = p.pairs + ((long long)b * N + s_path[j0 + warp]) * p.n_chunks;
       float tau = -INFINITY;
       if (p.n_chunks >= K) {
         unsigned long long below = ~0ull;
         for (int r = 0; r < K; ++r) {
           unsigned long long best = 0ull;
           for (int ch = lane; ch < p.n_chunks; ch += 32) {
-            const unsigned long long key = select_key(__float_as_uint(s_cmax[ch]), (uint32_t)ch);
+            const unsigned long long key = select_key(__float_as_uint(pairs[ch].y), (uint32_t)ch);
             if (key < below && key > best) best = key;
           }
           below = warp_max_u64(best);
         }
         tau = key_value(below);
       }
-      if (lane == 0) s_floor = tau;
+      if (lane == 0) s_floor[warp] = tau;
+      for (int ch = lane; ch < p.n_chunks; ch += 32)
+        if (pairs[ch].y >= tau) {
+          const int pos = atomicAdd(&s_nitems, 1);
+          if (pos < TOPK_ITEMS) s_items[pos] = ((uint32_t)warp << 16) | (uint32_t)ch;
+        }
     }
     __syncthreads();
-    const float floor = s_floor;
-    for (int ch = tid; ch < p.n_chunks; ch += K2_THREADS)
-      if (s_cmax[ch] >= floor) s_qlist[atomicAdd(&s_nq, 1)] = (unsigned short)ch;
+    const bool items_over = s_nitems > TOPK_ITEMS;
+    const int nitems = items_over ? 0 : s_nitems;
+    for (int it = warp; it < nitems; it += K2_THREADS / 32) {
+      const uint32_t item = s_items[it];
+      const int r = (int)(item >> 16), ch = (int)(item & 0xFFFFu);
+      push_chunk_candidates(p.logits, p.dtype, (long long)b * N + s_path[j0 + r], p.V, ch, s_floor[r], wide, s_cand[r],
+                            &s_ncand[r], CAND_CAP, lane);
+    }
     __syncthreads();
-    const int nq = s_nq;
-    for (int qi = warp; qi < nq; qi += K2_THREADS / 32)
-      push_chunk_candidates(p.logits, p.dtype, row, p.V, (int)s_qlist[qi], floor, wide, s_cand, &s_ncand, BLOCK_CANDS, lane);
-    __syncthreads();
-    if (warp == 0) {
-      int n = s_ncand;
-      if (n > BLOCK_CANDS) {
-        // more entries reach the bound than the buffer holds (long runs of equal values): the streaming
+    if (warp < nr) {
+      const int j = j0 + warp, u = s_path[j];
+      const long long row = (long long)b * N + u;
+      int n = s_ncand[warp];
+      if (items_over || n > CAND_CAP) {
+        // more entries reach the bound than the buffers hold (long runs of equal values): the streaming
         // selection copes with any input, one chunk at a time
-        n = row_topk_warp(p.logits, p.dtype, row, p.V, pairs, p.n_chunks, K, s_cand, &s_ncand, lane);
+        n = row_topk_warp(p.logits, p.dtype, row, p.V, p.pairs + row * p.n_chunks, p.n_chunks, K, s_cand[warp],
+                          &s_ncand[warp], lane);
       } else {
-        if (n > 0) compact_topk(s_cand, &s_ncand, n, K, lane, floor);
+        if (n > 0) compact_topk(s_cand[warp], &s_ncand[warp], n, K, lane, s_floor[warp]);
         n = n < K ? n : K;
       }
       if (lane < K) {
         const long long at = ((long long)b * W1 + j) * K + lane;
         if (lane < n) {
-          const uint2 e = s_cand[lane];
+          const uint2 e = s_cand[warp][lane];
           p.rec_ids[at] = (int)e.y;
-          p.rec_p[at] = (float)(exp2((double)__uint_as_float(e.x) * cd - (double)s_off[u]) / s_Z[u]);
+          p.rec_p[at] = (float)(exp2_d((double)__uint_as_float(e.x) * cd - (double)s_off[u]) / s_Z[u]);
         } else {
           p.rec_ids[at] = -1;
           p.rec_p[at] = 0.0f;
