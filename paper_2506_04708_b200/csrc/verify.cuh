@@ -6,7 +6,7 @@
 //   phase 1 (all warps)  normaliser of every row of the sequence from the chunk
 //                        pairs (8 lanes per row), and the target probability of every
 //                        drafted candidate (one round of gathered logits);
-//   phase 2 (thread 0)   the walk: children in draft order, accept iff
+//   phase 2 (warp 0)     the walk: children in draft order, accept iff
 //                        U * q(x) < p~(x); on rejection p~ <- norm(max(0, p~ - q)),
 //                        x leaves q; off the candidate list p~ is the target scaled
 //                        by a running factor, so the residual needs no pass over V;
@@ -127,7 +127,61 @@ __device__ __forceinline__ void push_chunk_candidates(const void* logits, int dt
   }
 }
 
-__global__ void __launch_bounds__(K2_THREADS) verify_kernel(const VerifyParams p) {
+// The same for rows whose entries can be read as aligned 16-byte vectors, split in two so that the loads
+// of several chunks are in flight before any of them is examined.  DT: 0 float (8 vectors per lane and
+// chunk), 1 bfloat16 (4 vectors).
+template <int DT>
+__device__ __forceinline__ void load_chunk_wide(const void* logits, long long row, int V, int ch, int lane,
+                                                uint4 (&v)[DT == 1 ? 4 : 8]) {
+  constexpr int NV = DT == 1 ? 4 : 8, VEC = DT == 1 ? 8 : 4;
+  const uint32_t fill = DT == 1 ? 0xFF80FF80u : 0xFF800000u;
+  const char* base = (const char*)logits + (size_t)row * (size_t)V * (DT == 1 ? 2 : 4);
+#pragma unroll
+  for (int k = 0; k < NV; ++k) {
+    const int i0 = ch * CHUNK + (k * 32 + lane) * VEC;
+    v[k] = i0 < V ? __ldg(reinterpret_cast<const uint4*>(base + (size_t)i0 * (DT == 1 ? 2 : 4))) : make_uint4(fill, fill, fill, fill);
+  }
+}
+template <int DT>
+__device__ __forceinline__ void push_chunk_wide(const uint4 (&v)[DT == 1 ? 4 : 8], int V, int ch, float floor, uint2* buf,
+                                                int* cnt, int cap, int lane) {
+  constexpr int NV = DT == 1 ? 4 : 8, VEC = DT == 1 ? 8 : 4;
+#pragma unroll
+  for (int k = 0; k < NV; ++k) {
+    float f[VEC];
+    ElemTraits<DT>::unpack(v[k], f);
+    const int i0 = ch * CHUNK + (k * 32 + lane) * VEC;
+    if (ElemTraits<DT>::vmax(v[k]) >= floor) {
+#pragma unroll
+      for (int e = 0; e < VEC; ++e) {
+        if (f[e] >= floor && i0 + e < V) {
+          const int pos = atomicAdd(cnt, 1);
+          const float canon = f[e] == 0.0f ? 0.0f : f[e];  // -0 and +0 are one value
+          if (pos < cap) buf[pos] = make_uint2(__float_as_uint(canon), (uint32_t)(i0 + e));
+        }
+      }
+    }
+  }
+}
+// Work items it, it + stride, ... of the list, two at a time.
+template <int DT>
+__device__ __forceinline__ void scan_items_wide(const void* logits, const int* path, long long row0, int V,
+                                                const uint32_t* items, int nitems, int first, int stride,
+                                                const float* floors, uint2 (*cand)[CAND_CAP], int* ncand, int lane) {
+  constexpr int NV = DT == 1 ? 4 : 8;
+  for (int it = first; it < nitems; it += 2 * stride) {
+    const bool two = it + stride < nitems;
+    const uint32_t a = items[it], c = items[two ? it + stride : it];
+    const int ra = (int)(a >> 16), cha = (int)(a & 0xFFFFu), rc = (int)(c >> 16), chc = (int)(c & 0xFFFFu);
+    uint4 va[NV], vc[NV];
+    load_chunk_wide<DT>(logits, row0 + path[ra], V, cha, lane, va);
+    if (two) load_chunk_wide<DT>(logits, row0 + path[rc], V, chc, lane, vc);
+    push_chunk_wide<DT>(va, V, cha, floors[ra], cand[ra], &ncand[ra], CAND_CAP, lane);
+    if (two) push_chunk_wide<DT>(vc, V, chc, floors[rc], cand[rc], &ncand[rc], CAND_CAP, lane);
+  }
+}
+
+__global__ void __launch_bounds__(K2_THREADS, 2) verify_kernel(const VerifyParams p) {
   __shared__ float s_off[NODES_MAX];
   __shared__ double s_Z[NODES_MAX];
   __shared__ double s_p[NODES_MAX][KMAX];  // target probability of candidate i of node u
@@ -146,7 +200,6 @@ __global__ void __launch_bounds__(K2_THREADS) verify_kernel(const VerifyParams p
   __shared__ double s_scale;         // residual target off the candidates = scale * target
   __shared__ int s_pick, s_pick_last;
   __shared__ double s_base;
-  __shared__ double s_q[KMAX], s_pt[KMAX];  // the walk's draft and residual target distributions
   // top-k selection of up to TOPK_ROWS path rows at a time
   __shared__ uint32_t s_items[TOPK_ITEMS];  // (row slot << 16) | chunk: chunks that can hold a top-k entry
   __shared__ uint2 s_cand[TOPK_ROWS][CAND_CAP];
@@ -173,7 +226,17 @@ __global__ void __launch_bounds__(K2_THREADS) verify_kernel(const VerifyParams p
   if (tid < p.n_max) s_tail[tid] = p.tail[b * p.n_max + tid];
   __syncthreads();
 
-  // ---- phase 1: normalisers (8 lanes per row), then all candidate logits in one round of gathers ----
+  // ---- phase 1: the candidate logits are requested first (one round of gathers), the normalisers
+  // (8 lanes per row) are formed while they travel ----
+  constexpr int GATHERS = NODES_MAX * KMAX / K2_THREADS;
+  float gx[GATHERS];
+#pragma unroll
+  for (int k = 0; k < GATHERS; ++k) {
+    const int i = tid + k * K2_THREADS;
+    const int u = i / KMAX, t = i - u * KMAX;
+    gx[k] = 0.0f;
+    if (u < N && t < s_cn[u]) gx[k] = load_logit(p.logits, p.dtype, ((long long)b * N + u) * (long long)p.V + s_cid[u][t]);
+  }
   {
     const int gl = tid & (ROW_LANES - 1);
     for (int u0 = 0; u0 < N; u0 += K2_THREADS / ROW_LANES) {
@@ -197,74 +260,71 @@ __global__ void __launch_bounds__(K2_THREADS) verify_kernel(const VerifyParams p
     }
   }
   __syncthreads();
-  for (int i = tid; i < N * KMAX; i += K2_THREADS) {
+#pragma unroll
+  for (int k = 0; k < GATHERS; ++k) {
+    const int i = tid + k * K2_THREADS;
     const int u = i / KMAX, t = i - u * KMAX;
-    if (t < s_cn[u]) {
-      const float x = load_logit(p.logits, p.dtype, ((long long)b * N + u) * (long long)p.V + s_cid[u][t]);
-      s_p[u][t] = exp2_d((double)x * cd - (double)s_off[u]) / s_Z[u];
-    }
+    if (u < N && t < s_cn[u]) s_p[u][t] = exp2_d((double)gx[k] * cd - (double)s_off[u]) / s_Z[u];
   }
   __syncthreads();
 
-  // ---- phase 2: the walk -----------------------------------------------------
-  if (tid == 0) {
+  // ---- phase 2: the walk, by warp 0: lane i carries candidate i of the current node ---------------
+  if (warp == 0) {
     int u = 0, m = 0;
-    s_path[0] = 0;
     int nsup = 0;
     double scale = 1.0;
+    if (lane == 0) s_path[0] = 0;
     for (;;) {
       const int fc = s_fc[u], nch = s_nch[u];
-      int drafted = 0;
-      while (drafted < nch && s_tree[fc + drafted] >= 0) ++drafted;
+      // children are drafted in rank order: count the leading drafted ones
+      const unsigned have = __ballot_sync(FULL, lane < nch && s_tree[fc + (lane < nch ? lane : 0)] >= 0);
+      const int drafted = __ffs(~have) - 1;
       nsup = 0;
       scale = 1.0;
       if (drafted == 0) break;  // nothing drafted below u: sample from its target
       const int nc = s_cn[u];
-      double phis = 0.0;
-      for (int i = 0; i < nc; ++i) phis += (double)s_cphi[u][i];
-      const double inv_phis = 1.0 / phis;
-      for (int i = 0; i < nc; ++i) { s_q[i] = (double)s_cphi[u][i] * inv_phis; s_pt[i] = s_p[u][i]; }
+      const int cid = lane < nc ? s_cid[u][lane] : -1;
+      double pt = lane < nc ? s_p[u][lane] : 0.0;
+      double q = lane < nc ? (double)s_cphi[u][lane] : 0.0;
+      q *= 1.0 / warp_sum_d(q);
+      // the uniforms of all children at once
+      const double Uj = lane < drafted ? (double)philox_u24(p.seed, b, p.step, u, (uint32_t)lane) * (1.0 / 16777216.0) : 0.0;
       int accepted = -1;
       for (int j = 0; j < drafted; ++j) {
         const int x = s_tree[fc + j];
-        int ix = -1;
-        for (int i = 0; i < nc; ++i)
-          if (s_cid[u][i] == x) ix = i;
-        const double U = (double)philox_u24(p.seed, b, p.step, u, (uint32_t)j) * (1.0 / 16777216.0);
-        if (ix < 0 || U * s_q[ix] < s_pt[ix]) { accepted = j; break; }
-        // rejected: residual target, x leaves the draft distribution
-        double overlap = 0.0;
-        for (int i = 0; i < nc; ++i) overlap += fmin(s_pt[i], s_q[i]);
-        const double inv_zr = 1.0 / (1.0 - overlap);
-        double qs = 0.0;
-        for (int i = 0; i < nc; ++i) {
-          const double qi = s_q[i];
-          s_pt[i] = fmax(0.0, s_pt[i] - qi) * inv_zr;
-          if (i != ix) qs += qi;
-        }
-        s_q[ix] = 0.0;
+        const unsigned hit = __ballot_sync(FULL, lane < nc && cid == x);
+        const int ix = hit ? 31 - __clz(hit) : -1;
+        const double U = __shfl_sync(FULL, Uj, j);
+        const double qx = __shfl_sync(FULL, q, ix < 0 ? 0 : ix);
+        const double ptx = __shfl_sync(FULL, pt, ix < 0 ? 0 : ix);
+        if (ix < 0 || U * qx < ptx) { accepted = j; break; }
+        // rejected: residual target norm(max(0, p~ - q)); x leaves the draft distribution, whose
+        // remaining mass is 1 - q(x)
+        const double inv_zr = 1.0 / (1.0 - warp_sum_d(fmin(pt, q)));
+        pt = fmax(0.0, pt - q) * inv_zr;
         scale *= inv_zr;
-        if (qs > 0.0) {
-          const double inv_qs = 1.0 / qs;
-          for (int i = 0; i < nc; ++i) s_q[i] *= inv_qs;
-        }
+        if (lane == ix) q = 0.0;
+        const double rest = 1.0 - qx;
+        q = rest > 0.0 ? q * (1.0 / rest) : 0.0;
       }
       if (accepted >= 0) {
-        s_emit[m] = s_tree[fc + accepted];
+        if (lane == 0) s_emit[m] = s_tree[fc + accepted];
         u = fc + accepted;
         ++m;
-        s_path[m] = u;
+        if (lane == 0) s_path[m] = u;
         continue;
       }
       nsup = nc;
-      for (int i = 0; i < nc; ++i) { s_sup_id[i] = s_cid[u][i]; s_sup_pt[i] = s_pt[i]; s_sup_p[i] = s_p[u][i]; }
+      if (lane < nc) { s_sup_id[lane] = cid; s_sup_pt[lane] = pt; s_sup_p[lane] = s_p[u][lane]; }
       break;
     }
-    s_m = m;
-    s_nsup = nsup;
-    s_scale = scale;
-    s_pick = 0x7FFFFFFF;
-    s_pick_last = -1;
+    if (lane == 0) {
+      s_m = m;
+      s_nsup = nsup;
+      s_scale = scale;
+      s_pick = 0x7FFFFFFF;
+      s_pick_last = -1;
+    }
   }
   __syncthreads();
 
@@ -428,12 +488,19 @@ __global__ void __launch_bounds__(K2_THREADS) verify_kernel(const VerifyParams p
     __syncthreads();
     const bool items_over = s_nitems > TOPK_ITEMS;
     const int nitems = items_over ? 0 : s_nitems;
-    for (int it = warp; it < nitems; it += K2_THREADS / 32) {
-      const uint32_t item = s_items[it];
-      const int r = (int)(item >> 16), ch = (int)(item & 0xFFFFu);
-      push_chunk_candidates(p.logits, p.dtype, (long long)b * N + s_path[j0 + r], p.V, ch, s_floor[r], wide, s_cand[r],
-                            &s_ncand[r], CAND_CAP, lane);
-    }
+    if (wide && p.dtype == 1)
+      scan_items_wide<1>(p.logits, s_path + j0, (long long)b * N, p.V, s_items, nitems, warp, K2_THREADS / 32, s_floor, s_cand,
+                         s_ncand, lane);
+    else if (wide)
+      scan_items_wide<0>(p.logits, s_path + j0, (long long)b * N, p.V, s_items, nitems, warp, K2_THREADS / 32, s_floor, s_cand,
+                         s_ncand, lane);
+    else
+      for (int it = warp; it < nitems; it += K2_THREADS / 32) {
+        const uint32_t item = s_items[it];
+        const int r = (int)(item >> 16), ch = (int)(item & 0xFFFFu);
+        push_chunk_candidates(p.logits, p.dtype, (long long)b * N + s_path[j0 + r], p.V, ch, s_floor[r], false, s_cand[r],
+                              &s_ncand[r], CAND_CAP, lane);
+      }
     __syncthreads();
     if (warp < nr) {
       const int j = j0 + warp, u = s_path[j];
