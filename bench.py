@@ -23,7 +23,7 @@ ROOT = os.path.dirname(os.path.abspath(__file__))
 if ROOT not in sys.path:
     sys.path.insert(0, ROOT)
 
-from paper_2506_04708_b200 import inputs  # noqa: E402
+from paper_2506_04708_b200 import dist as sd, inputs  # noqa: E402
 
 METRIC = "draft-tree nodes verified/sec at V=151,936 bf16"
 UNIT = "nodes/s"
@@ -118,6 +118,65 @@ def workload_of(args):
     return w
 
 
+# DRAM bytes per row-pass launch from the ncu capture summarised in profiles/row_pass_kernel_cfg5_B64_ncu_full.md
+# (dram__bytes_read.sum + dram__bytes_write.sum = 466.77 MB + 5.2 MB at B=64; traffic grows with the rows, so a
+# launch over B sequences moves B/64 times that).  None for shapes that were not captured.
+ROW_PASS_TRAFFIC_PER_SEQUENCE = {"cfg5": (466.77e6 + 5.2e6) / 64}
+
+
+def quick_workload(name, args, dev, peaks):
+    """A short closed-loop run of one of the other workloads: nodes/s and logits GB/s (device-timed, warm)."""
+    import torch
+    from paper_2506_04708_b200.binding import Stand
+    w = inputs.WORKLOADS[name]
+    parent = inputs.topology(w.N, w.D, w.kb)
+    depth = inputs.node_depths(parent)
+    esize = 2 if w.dtype == inputs.DTYPE_BF16 else 4
+    step_bytes = w.B * w.N * w.V * esize
+    ring_n = min(512, max(4, -(-3 * L2_BYTES // step_bytes)))
+    steps = max(200, min(2000, int(0.25 / (step_bytes / 5e12 + 40e-6))))
+    gpu = Stand(w.B, w.N, w.V, w.topk, w.order_max, w.dtype, w.T, args.seed, min(w.table_slots, 1 << 22), parent, device=dev)
+    prompt = 8
+    streams = inputs.token_streams(w, args.seed, prompt + (ring_n + 4) * (w.D + 2))
+    tail = np.ascontiguousarray(streams[:, prompt - w.order_max:prompt])
+    gpu.reset_sequences(torch.from_numpy(tail), torch.full((w.B,), prompt, dtype=torch.int64))
+    gen = inputs.DeviceLogits(w, streams, depth, args.seed, pool=2, device=dev, peak_mode=args.peak_mode)
+    tdtype = torch.bfloat16 if w.dtype == inputs.DTYPE_BF16 else torch.float32
+    ring = [torch.empty((w.B, w.N, w.V), dtype=tdtype, device=dev) for _ in range(ring_n)]
+    lens = torch.empty(w.B, dtype=torch.int64, device=dev)
+    for s in range(ring_n):
+        gpu.lens_device(lens)
+        gen.make(ring[s], lens, s)
+        gpu.step(ring[s])
+    for s in range(5):
+        gpu.step(ring[s % ring_n])
+    ev0, ev1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    torch.cuda.synchronize()
+    ev0.record()
+    for s in range(steps):
+        gpu.step(ring[s % ring_n])
+    ev1.record()
+    torch.cuda.synchronize()
+    ms = ev0.elapsed_time(ev1) / steps
+    sev = [torch.cuda.Event(enable_timing=True) for _ in range(5)]
+    for e in sev:
+        e.record()
+    k1 = []
+    for s in range(20):
+        gpu.profile_stages(sev)
+        gpu.step(ring[s % ring_n])
+        torch.cuda.synchronize()
+        k1.append(sev[0].elapsed_time(sev[1]))
+    gpu.profile_stages(None)
+    st = gpu.stats()
+    gpu.close()
+    k1_ms = statistics.median(k1)
+    return {"workload": describe(w), "steps": steps, "ring_buffers": ring_n, "ms_per_step": ms,
+            "nodes_per_s": w.B * w.N / (ms * 1e-3), "logits_gbs": step_bytes / (ms * 1e-3) / 1e9,
+            "row_pass_us": k1_ms * 1e3, "row_pass_gbs": step_bytes / (k1_ms * 1e-3) / 1e9,
+            "row_pass_frac_of_measured": step_bytes / (k1_ms * 1e-3) / 1e9 / peaks["hbm_gbs"], "drops": st["drops"]}
+
+
 def run_ours(args, rank, world, local):
     import torch
     from paper_2506_04708_b200.binding import Stand
@@ -125,11 +184,8 @@ def run_ours(args, rank, world, local):
     w = workload_of(args)
     dev = torch.device("cuda", local)
     torch.cuda.set_device(dev)
-    dist = None
-    if world > 1:
-        import torch.distributed as dist
-        dist.init_process_group("nccl", device_id=dev)
-    seed = args.seed + 7919 * rank  # every rank runs its own sequences: independent replicas
+    dist = sd.init("nccl", dev)
+    seed = sd.replica_seed(args.seed, rank)  # every rank runs its own sequences: independent replicas
     parent = inputs.topology(w.N, w.D, w.kb)
     depth = inputs.node_depths(parent)
     esize = 2 if w.dtype == inputs.DTYPE_BF16 else 4
@@ -217,13 +273,10 @@ def run_ours(args, rank, world, local):
                 for i, name in enumerate(("row_pass", "verify", "update", "draft"))}
     clocks = sampler.stop()
 
-    if dist is not None:
-        t = torch.tensor([ms_total], dtype=torch.float64, device=dev)
-        dist.all_reduce(t, op=dist.ReduceOp.MAX)
-        ms_total = float(t.item())
+    ms_total = sd.max_over_ranks(dist, ms_total, dev)
     ms_per_step = ms_total / args.steps
     nodes_per_step = w.B * w.N * world
-    value = nodes_per_step / (ms_per_step * 1e-3)
+    value = sd.whole_job_rate(w.B * w.N, world, args.steps, ms_total)
 
     # ---- end to end through the C ABI with host buffers ---------------------------------
     e2e_steps = max(2, min(8, int(4e9 // step_bytes) or 2))
@@ -239,10 +292,7 @@ def run_ours(args, rank, world, local):
         gpu.step_host(h_logits, h_em, h_ne, h_tr)
     barrier()
     e2e_s = time.perf_counter() - t0
-    if dist is not None:
-        t = torch.tensor([e2e_s], dtype=torch.float64, device=dev)
-        dist.all_reduce(t, op=dist.ReduceOp.MAX)
-        e2e_s = float(t.item())
+    e2e_s = sd.max_over_ranks(dist, e2e_s, dev)
     e2e = {"value": nodes_per_step * e2e_steps / e2e_s, "unit": UNIT, "steps": e2e_steps,
            "h2d_bytes_per_step": step_bytes, "d2h_bytes_per_step": (h_em.numel() + h_ne.numel() + h_tr.numel()) * 4}
 
@@ -253,14 +303,25 @@ def run_ours(args, rank, world, local):
                 "unit": "GB/s", "frac": achieved / peaks["hbm_gbs"], "peak_kind": peak_kind + " copy bandwidth",
                 "traffic": None, "kernel_ms": k1_ms, "frac_of_nominal_8TBs": achieved / 8000.0,
                 "step_frac": alg_bytes / (ms_per_step * 1e-3) / 1e9 / peaks["hbm_gbs"]}
-    prof = os.path.join(ROOT, "profiles", f"traffic_{w.name}.json")
-    if os.path.exists(prof):
-        with open(prof) as f:
-            roofline["traffic"] = json.load(f).get("dram_bytes_per_launch")
+    if args.workload in ROW_PASS_TRAFFIC_PER_SEQUENCE:
+        roofline["traffic"] = ROW_PASS_TRAFFIC_PER_SEQUENCE[args.workload] * w.B
+        roofline["traffic_source"] = "ncu capture at B=64 scaled by rows (profiles/row_pass_kernel_cfg5_B64_ncu_full.md)"
+    roofline["algorithmic_bytes"] = alg_bytes
 
     cpu_baseline = None
     if rank == 0 and world == 1 and not args.no_cpu_baseline:
         cpu_baseline = time_oracle(w, ring[0], args, total_budget_s=12.0)
+
+    others = None
+    if rank == 0 and world == 1 and not args.no_sweep:
+        # the other four workloads, briefly (secondary figures; the line's value is the named workload's)
+        del ring, h_logits
+        torch.cuda.empty_cache()
+        others = {}
+        for name in sorted(inputs.WORKLOADS):
+            if name != args.workload:
+                others[name] = quick_workload(name, args, dev, peaks)
+                torch.cuda.empty_cache()
 
     if rank == 0:
         line = {
@@ -280,6 +341,8 @@ def run_ours(args, rank, world, local):
         }
         if cpu_baseline is not None:
             line["cpu_baseline"] = cpu_baseline
+        if others is not None:
+            line["other_workloads"] = others
         print(json.dumps(line))
     gpu.close()
     if dist is not None:
@@ -358,12 +421,11 @@ def main():
     ap.add_argument("--peak-mode", default="add8", choices=["add8", "p80"])
     ap.add_argument("--seed", type=int, default=0)
     ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--no-sweep", action="store_true", help="skip the short runs of the other four workloads")
     ap.add_argument("--batch", type=int, default=0, help="override the workload's number of sequences (profiling)")
     ap.add_argument("--ring", type=int, default=0, help="override the number of logit buffers in the ring (profiling)")
     args = ap.parse_args()
-    rank = int(os.environ.get("RANK", "0"))
-    world = int(os.environ.get("WORLD_SIZE", "1"))
-    local = int(os.environ.get("LOCAL_RANK", "0"))
+    rank, world, local = sd.env_ranks()
     if args.impl == "reference":
         run_reference(args, rank, world)
     else:

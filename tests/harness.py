@@ -67,7 +67,8 @@ def resync_gpu_from_oracle(gpu, orc):
 class ClosedLoop:
     """Runs the same seeded workload through both sides, step by step."""
 
-    def __init__(self, w, seed=0, peak_mode="add8", table_slots=None, prompt=8, device="cuda:0", **stand_kw):
+    def __init__(self, w, seed=0, peak_mode="add8", table_slots=None, prompt=8, device="cuda:0", device_logits=False,
+                 **stand_kw):
         from paper_2506_04708_b200.binding import Stand
         self.w, self.seed, self.peak_mode = w, seed, peak_mode
         self.parent = inputs.topology(w.N, w.D, w.kb)
@@ -84,6 +85,14 @@ class ClosedLoop:
         self.lens = np.full(w.B, prompt, np.int64)
         self.gpu.reset_sequences(torch.from_numpy(tail), torch.from_numpy(self.lens))
         self.orc.reset_sequences(tail, self.lens)
+        self.gen = None
+        if device_logits:
+            # full-size workloads: the logits are made on the device (as the benchmark does) and copied to the host
+            # for the oracle; both sides still see the same bytes
+            self.gen = inputs.DeviceLogits(w, self.streams, self.depth, seed, pool=1, device=self.gpu.dev,
+                                           peak_mode=peak_mode)
+            tdtype = torch.bfloat16 if w.dtype == inputs.DTYPE_BF16 else torch.float32
+            self.dev_buf = torch.empty((w.B, w.N, w.V), dtype=tdtype, device=self.gpu.dev)
         self.step_no = 0
         self.tolerated = 0
         self.emitted_total = 0
@@ -92,8 +101,14 @@ class ClosedLoop:
 
     def step(self):
         w = self.w
-        logits = inputs.logits_numpy(w, self.streams, self.lens, self.depth, self.step_no, self.seed, self.peak_mode)
-        dl = to_device_logits(logits, self.gpu.dev)
+        if self.gen is not None:
+            import torch
+            dl = self.gen.make(self.dev_buf, torch.from_numpy(np.asarray(self.lens, np.int64)).to(self.gpu.dev), self.step_no)
+            host = dl.cpu()
+            logits = host.view(torch.int16).numpy().view(np.uint16) if w.dtype == inputs.DTYPE_BF16 else host.numpy()
+        else:
+            logits = inputs.logits_numpy(w, self.streams, self.lens, self.depth, self.step_no, self.seed, self.peak_mode)
+            dl = to_device_logits(logits, self.gpu.dev)
         em_g, ne_g, tr_g = (t.cpu().numpy() for t in self.gpu.step(dl))
         em_o, ne_o, tr_o = self.orc.step(logits)
         ints, margins = self.orc.take_margins()

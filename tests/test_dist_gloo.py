@@ -1,0 +1,59 @@
+"""The N > 1 path of the benchmark on CPU: two gloo ranks, independent replicas, max-over-ranks timing."""
+import json
+import os
+import subprocess
+import sys
+
+import pytest
+import torch.multiprocessing as mp
+
+from paper_2506_04708_b200 import dist as sd, inputs
+
+ROOT = os.path.dirname(os.path.dirname(os.path.abspath(__file__)))
+
+
+def _worker(rank, world, port, out_dir):
+    os.environ.update(RANK=str(rank), WORLD_SIZE=str(world), LOCAL_RANK=str(rank), MASTER_ADDR="127.0.0.1",
+                      MASTER_PORT=str(port))
+    assert sd.env_ranks() == (rank, world, rank)
+    d = sd.init("gloo")
+    assert d is not None and d.get_world_size() == world
+    sd.barrier(d)
+    # every rank "measured" a different time: all of them learn the slowest one
+    mine = 10.0 + 5.0 * rank
+    slowest = sd.max_over_ranks(d, mine)
+    # replicas are independent: different seeds give different streams
+    w = inputs.scaled(inputs.WORKLOADS["cfg1"], B=2)
+    s = inputs.token_streams(w, sd.replica_seed(0, rank), 64)
+    res = {"rank": rank, "slowest": slowest, "stream_head": s[0, :8].tolist(),
+           "rate": sd.whole_job_rate(w.B * w.N, world, 100, slowest)}
+    with open(os.path.join(out_dir, f"r{rank}.json"), "w") as f:
+        json.dump(res, f)
+    sd.barrier(d)
+    d.destroy_process_group()
+
+
+def test_two_gloo_ranks_agree_on_the_slowest_time(tmp_path):
+    world, port = 2, 29000 + os.getpid() % 2000
+    mp.spawn(_worker, args=(world, port, str(tmp_path)), nprocs=world, join=True)
+    r = [json.load(open(tmp_path / f"r{k}.json")) for k in range(world)]
+    assert r[0]["slowest"] == r[1]["slowest"] == 15.0
+    assert r[0]["stream_head"] != r[1]["stream_head"]
+    # 2 ranks x (2 sequences x 8 nodes) x 100 steps over 15 ms
+    assert r[0]["rate"] == pytest.approx(2 * 16 * 100 / 15e-3)
+
+
+def test_single_process_needs_no_group():
+    os.environ.pop("WORLD_SIZE", None)
+    os.environ.pop("RANK", None)
+    assert sd.env_ranks()[1] == 1
+    assert sd.init("gloo") is None
+    assert sd.max_over_ranks(None, 3.5) == 3.5
+    assert sd.replica_seed(5, 0) == 5 and sd.replica_seed(5, 3) != sd.replica_seed(5, 2)
+
+
+def test_reference_arm_runs_on_rank_zero_only():
+    env = dict(os.environ, RANK="1", WORLD_SIZE="2", LOCAL_RANK="1")
+    out = subprocess.run([sys.executable, os.path.join(ROOT, "bench.py"), "--impl", "reference", "--gpus", "2", "--steps", "1",
+                          "--warmup", "0"], env=env, capture_output=True, text=True, timeout=120)
+    assert out.returncode == 0 and out.stdout.strip() == ""

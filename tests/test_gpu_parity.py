@@ -69,7 +69,7 @@ def _run(w, steps, peak_mode, seed=0, check_every=0, **kw):
         assert loop.hard == [], loop.hard[:3]
         assert loop.check_state_and_table() == []
         st = loop.gpu.stats()
-        assert st["drops"] == 0 and st["bad_tokens"] == 0
+        assert st["drops"] == 0 and st["bad_tokens"] == 0 and st["wait_timeouts"] == 0
         # a handful of low-margin decisions at most
         assert loop.tolerated <= max(2, steps // 100)
         return loop.emitted_total / (steps * w.B), loop.tolerated, st
@@ -103,6 +103,26 @@ def test_cfg5_shape_small_vocab():
     # the tree-search shape (256 forked beams, shared prefixes -> many same-step updates of one context)
     w = inputs.scaled(inputs.WORKLOADS["cfg5"], V=4096)
     _run(w, 40, "p80", table_slots=1 << 18, check_every=10)
+
+
+@pytest.mark.parametrize("peak_mode", ["add8", "p80"])
+def test_cfg5_full_size_in_the_benchmark_configuration(peak_mode):
+    """The benchmark's workload at full size (256 x 24 rows of 151,936 bf16, 16M-slot table): whole steps against the
+    oracle, every emitted token, tree, table entry and state word."""
+    w = inputs.WORKLOADS["cfg5"]
+    steps = 4
+    loop = harness.ClosedLoop(inputs.scaled(w, steps=steps), seed=0, peak_mode=peak_mode, device_logits=True)
+    try:
+        for _ in range(steps):
+            loop.step()
+        assert loop.hard == [], loop.hard[:3]
+        assert loop.check_state_and_table() == []
+        st = loop.gpu.stats()
+        assert st["drops"] == 0 and st["bad_tokens"] == 0 and st["wait_timeouts"] == 0
+        assert st["records"] >= w.B * steps
+        assert loop.tolerated <= 2
+    finally:
+        loop.close()
 
 
 @pytest.mark.parametrize("V,N,D,kb", [(16, 1, 0, 1), (13, 4, 2, 2), (50, 7, 3, 2), (1000, 16, 4, 3)])
