@@ -133,10 +133,14 @@ __global__ void __launch_bounds__(K4_THREADS) draft_kernel(const DraftParams p) 
       const uint32_t u24 = valid ? philox_u24(p.seed, b, p.step, u, SLOT_GUMBEL | (uint32_t)id) : 0u;
       float gf = 0.0f;
       if (valid) {
-        // -log U with U = (u24 + 1/2) / 2^24: above one half through log1p of the exact complement
-        const float L = u24 < (1u << 23) ? -logf(((float)u24 + 0.5f) * (1.0f / 16777216.0f))
-                                         : -log1pf(-((float)(16777216u - u24) - 0.5f) * (1.0f / 16777216.0f));
-        gf = logf(phi) - logf(L);
+        // L = -log U with U = (u24 + 1/2) / 2^24.  Below one half U is exact in fp32 and the hardware
+        // logarithm serves; above, L = 2 atanh(v / (2 - v)) with the exact complement v = 1 - U <= 1/2.
+        const float lo = -__logf(((float)u24 + 0.5f) * (1.0f / 16777216.0f));
+        const float v = ((float)(16777216u - u24) - 0.5f) * (1.0f / 16777216.0f);
+        const float t = __fdividef(v, 2.0f - v), t2 = t * t;
+        const float hi = 2.0f * t * fmaf(t2, fmaf(t2, fmaf(t2, fmaf(t2, fmaf(t2, 1.0f / 11.0f, 1.0f / 9.0f), 1.0f / 7.0f), 0.2f), 1.0f / 3.0f), 1.0f);
+        const float L = u24 < (1u << 23) ? lo : hi;
+        gf = __logf(phi) - __logf(L);
       }
       int rank = 0;
       bool close = false;

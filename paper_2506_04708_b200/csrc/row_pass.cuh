@@ -350,27 +350,30 @@ struct RowNorm {
 };
 
 // All lanes of a warp call this; every lane gets the result.
+__device__ __forceinline__ RowNorm row_normaliser(const float2* pairs, int n_chunks, float c, int lane);
+
+// Mass of one chunk relative to the row offset `off` (before division by Z): s * 2^(o - off), exact in
+// fp32 (a power-of-two scaling; terms below 2^-126 of the row's largest flush to zero).
+__device__ __forceinline__ float chunk_mass_f(float2 pr, float c, float off) {
+  const int k = (int)(chunk_offset(pr.y, c) - off);
+  const float pw = k >= -126 ? __int_as_float((k + 127) << 23) : 0.0f;
+  return pr.x > 0.0f ? pr.x * pw : 0.0f;
+}
+__device__ __forceinline__ double chunk_mass(float2 pr, float c, float off) { return (double)chunk_mass_f(pr, c, off); }
+
+// All lanes of a warp call this; every lane gets the result.  The row offset is the offset of the largest
+// chunk maximum (the offset grows with the maximum).
 __device__ __forceinline__ RowNorm row_normaliser(const float2* pairs, int n_chunks, float c, int lane) {
-  float om = -INFINITY;
-  for (int ch = lane; ch < n_chunks; ch += 32) {
-    const float2 pr = pairs[ch];
-    if (pr.x > 0.0f) om = fmaxf(om, chunk_offset(pr.y, c));
-  }
-  om = warp_max_f(om);
+  float mm = -INFINITY;
+  for (int ch = lane; ch < n_chunks; ch += 32) mm = fmaxf(mm, pairs[ch].y);
+  mm = warp_max_f(mm);
+  const float om = chunk_offset(mm, c);
   double z = 0.0;
-  for (int ch = lane; ch < n_chunks; ch += 32) {
-    const float2 pr = pairs[ch];
-    if (pr.x > 0.0f) z += (double)pr.x * pow2_int((int)(chunk_offset(pr.y, c) - om));
-  }
+  for (int ch = lane; ch < n_chunks; ch += 32) z += (double)chunk_mass_f(pairs[ch], c, om);
   RowNorm r;
   r.off = om;
   r.Z = warp_sum_d(z);
   return r;
-}
-
-// Mass of one chunk relative to the row offset `off` (before division by Z).
-__device__ __forceinline__ double chunk_mass(float2 pr, float c, float off) {
-  return pr.x > 0.0f ? (double)pr.x * pow2_int((int)(chunk_offset(pr.y, c) - off)) : 0.0;
 }
 
 // Keeps the k best of the n buffered candidates at buf[0..k), best first; returns

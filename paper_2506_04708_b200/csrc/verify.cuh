@@ -181,9 +181,57 @@ __device__ __forceinline__ void scan_items_wide(const void* logits, const int* p
   }
 }
 
+// The k-th largest of a row's chunk maxima (a lower bound of the row's k-th largest entry); -inf when
+// the row has fewer than k chunks.  Called by all lanes of a warp.  Up to 256 chunks are held in
+// registers as order-preserving integers and the largest is removed k - 1 times through the integer
+// reduction unit; longer rows take the general loop.
+__device__ __forceinline__ float kth_largest_chunk_max(const float2* pairs, int n_chunks, int k, int lane) {
+  if (n_chunks < k) return -INFINITY;
+  if (n_chunks <= 256) {
+    uint32_t kv[8];  // 0 = no chunk (every real value maps above 0)
+#pragma unroll
+    for (int i = 0; i < 8; ++i) {
+      const int ch = lane + 32 * i;
+      kv[i] = ch < n_chunks ? ordered_bits(__float_as_uint(pairs[ch].y)) : 0u;
+    }
+    uint32_t mx = 0u;
+    for (int r = 0; r < k; ++r) {
+      uint32_t lm = kv[0];
+#pragma unroll
+      for (int i = 1; i < 8; ++i) lm = max(lm, kv[i]);
+      mx = warp_max_u32(lm);
+      const int owner = __ffs(__ballot_sync(FULL, lm == mx)) - 1;
+      if (lane == owner) {  // remove one instance
+        bool gone = false;
+#pragma unroll
+        for (int i = 0; i < 8; ++i)
+          if (!gone && kv[i] == mx) { kv[i] = 0u; gone = true; }
+      }
+    }
+    return __uint_as_float((mx & 0x80000000u) ? (mx ^ 0x80000000u) : ~mx);
+  }
+  unsigned long long below = ~0ull;
+  for (int r = 0; r < k; ++r) {
+    unsigned long long best = 0ull;
+    for (int ch = lane; ch < n_chunks; ch += 32) {
+      const unsigned long long key = select_key(__float_as_uint(pairs[ch].y), (uint32_t)ch);
+      if (key < below && key > best) best = key;
+    }
+    below = warp_max_u64(best);
+  }
+  return key_value(below);
+}
+
+// Sum over the 16 lanes of a half-warp (both halves carry the same values); every lane gets it.
+__device__ __forceinline__ double half_sum_d(double v) {
+#pragma unroll
+  for (int o = 8; o > 0; o >>= 1) v += __shfl_xor_sync(FULL, v, o);
+  return v;
+}
+
 __global__ void __launch_bounds__(K2_THREADS, 2) verify_kernel(const VerifyParams p) {
   __shared__ float s_off[NODES_MAX];
-  __shared__ double s_Z[NODES_MAX];
+  __shared__ double s_invZ[NODES_MAX];
   __shared__ double s_p[NODES_MAX][KMAX];  // target probability of candidate i of node u
   __shared__ int s_tree[NODES_MAX], s_cn[NODES_MAX], s_fc[NODES_MAX], s_nch[NODES_MAX];
   __shared__ int s_cid[NODES_MAX][KMAX];
@@ -243,20 +291,22 @@ __global__ void __launch_bounds__(K2_THREADS, 2) verify_kernel(const VerifyParam
       const int u = u0 + tid / ROW_LANES;
       const bool live = u < N;
       const float2* pairs = p.pairs + ((long long)b * N + (live ? u : 0)) * p.n_chunks;
-      float om = -INFINITY;
+      float mm = -INFINITY;
       if (live)
-        for (int ch = gl; ch < p.n_chunks; ch += ROW_LANES) {
-          const float2 pr = pairs[ch];
-          if (pr.x > 0.0f) om = fmaxf(om, chunk_offset(pr.y, p.c));
-        }
+        for (int ch = gl; ch < p.n_chunks; ch += ROW_LANES) mm = fmaxf(mm, pairs[ch].y);
 #pragma unroll
-      for (int o = ROW_LANES / 2; o > 0; o >>= 1) om = fmaxf(om, __shfl_xor_sync(FULL, om, o));
-      double z = 0.0;
+      for (int o = ROW_LANES / 2; o > 0; o >>= 1) mm = fmaxf(mm, __shfl_xor_sync(FULL, mm, o));
+      const float om = chunk_offset(mm, p.c);  // the offset grows with the maximum
+      double z0 = 0.0, z1 = 0.0;
       if (live)
-        for (int ch = gl; ch < p.n_chunks; ch += ROW_LANES) z += chunk_mass(pairs[ch], p.c, om);
+        for (int ch = gl; ch < p.n_chunks; ch += 2 * ROW_LANES) {
+          z0 += (double)chunk_mass_f(pairs[ch], p.c, om);
+          if (ch + ROW_LANES < p.n_chunks) z1 += (double)chunk_mass_f(pairs[ch + ROW_LANES], p.c, om);
+        }
+      double z = z0 + z1;
 #pragma unroll
       for (int o = ROW_LANES / 2; o > 0; o >>= 1) z += __shfl_xor_sync(FULL, z, o);
-      if (live && gl == 0) { s_off[u] = om; s_Z[u] = z; }
+      if (live && gl == 0) { s_off[u] = om; s_invZ[u] = 1.0 / z; }
     }
   }
   __syncthreads();
@@ -264,12 +314,20 @@ __global__ void __launch_bounds__(K2_THREADS, 2) verify_kernel(const VerifyParam
   for (int k = 0; k < GATHERS; ++k) {
     const int i = tid + k * K2_THREADS;
     const int u = i / KMAX, t = i - u * KMAX;
-    if (u < N && t < s_cn[u]) s_p[u][t] = exp2_d((double)gx[k] * cd - (double)s_off[u]) / s_Z[u];
+    if (u < N && t < s_cn[u]) s_p[u][t] = exp2_d((double)gx[k] * cd - (double)s_off[u]) * s_invZ[u];
   }
   __syncthreads();
 
-  // ---- phase 2: the walk, by warp 0: lane i carries candidate i of the current node ---------------
+  // ---- phase 2: the walk, by warp 0 ------------------------------------------------------------
+  // Lane i (and its mirror i + 16) carries candidate i of the current node.  Target and draft
+  // distributions are kept unnormalised with their normalisers, so a rejection costs one 16-lane sum
+  // and no division: with p~_i = ph_i / zr and q_i = qh_i / qn,
+  //   accept x        iff  U * qh_x * zr < ph_x * qn
+  //   after rejecting x:   ph_i <- max(0, ph_i * qn - qh_i * zr),  zr <- zr * qn - sum_i min(ph_i * qn, qh_i * zr),
+  //                        qh_x <- 0,  qn <- qn - qh_x
+  // and off the candidate list the residual target is the target times (product of the qn's) / zr.
   if (warp == 0) {
+    const int li = lane & 15;
     int u = 0, m = 0;
     int nsup = 0;
     double scale = 1.0;
@@ -281,31 +339,30 @@ __global__ void __launch_bounds__(K2_THREADS, 2) verify_kernel(const VerifyParam
       const int drafted = __ffs(~have) - 1;
       nsup = 0;
       scale = 1.0;
-      if (drafted == 0) break;  // nothing drafted below u: sample from its target
+      if (drafted <= 0) break;  // nothing drafted below u: sample from its target
       const int nc = s_cn[u];
-      const int cid = lane < nc ? s_cid[u][lane] : -1;
-      double pt = lane < nc ? s_p[u][lane] : 0.0;
-      double q = lane < nc ? (double)s_cphi[u][lane] : 0.0;
-      q *= 1.0 / warp_sum_d(q);
+      const int cid = li < nc ? s_cid[u][li] : -1;
+      double ph = li < nc ? s_p[u][li] : 0.0;
+      double qh = li < nc ? (double)s_cphi[u][li] : 0.0;
+      double qn = half_sum_d(qh), zr = 1.0, pq = 1.0;
       // the uniforms of all children at once
-      const double Uj = lane < drafted ? (double)philox_u24(p.seed, b, p.step, u, (uint32_t)lane) * (1.0 / 16777216.0) : 0.0;
+      const double Uj = li < drafted ? (double)philox_u24(p.seed, b, p.step, u, (uint32_t)li) * (1.0 / 16777216.0) : 0.0;
       int accepted = -1;
       for (int j = 0; j < drafted; ++j) {
         const int x = s_tree[fc + j];
-        const unsigned hit = __ballot_sync(FULL, lane < nc && cid == x);
+        const unsigned hit = __ballot_sync(FULL, li < nc && cid == x) & 0xFFFFu;
         const int ix = hit ? 31 - __clz(hit) : -1;
-        const double U = __shfl_sync(FULL, Uj, j);
-        const double qx = __shfl_sync(FULL, q, ix < 0 ? 0 : ix);
-        const double ptx = __shfl_sync(FULL, pt, ix < 0 ? 0 : ix);
-        if (ix < 0 || U * qx < ptx) { accepted = j; break; }
-        // rejected: residual target norm(max(0, p~ - q)); x leaves the draft distribution, whose
-        // remaining mass is 1 - q(x)
-        const double inv_zr = 1.0 / (1.0 - warp_sum_d(fmin(pt, q)));
-        pt = fmax(0.0, pt - q) * inv_zr;
-        scale *= inv_zr;
-        if (lane == ix) q = 0.0;
-        const double rest = 1.0 - qx;
-        q = rest > 0.0 ? q * (1.0 / rest) : 0.0;
+        const double U = __shfl_sync(FULL, Uj, j & 15);
+        const double qx = __shfl_sync(FULL, qh, ix < 0 ? 0 : ix);
+        const double px = __shfl_sync(FULL, ph, ix < 0 ? 0 : ix);
+        if (ix < 0 || U * qx * zr < px * qn) { accepted = j; break; }
+        const double a = ph * qn, c2 = qh * zr;
+        const double ov = half_sum_d(fmin(a, c2));
+        pq *= qn;
+        zr = zr * qn - ov;
+        ph = fmax(0.0, a - c2);
+        if (li == ix) qh = 0.0;
+        qn -= qx;
       }
       if (accepted >= 0) {
         if (lane == 0) s_emit[m] = s_tree[fc + accepted];
@@ -314,8 +371,10 @@ __global__ void __launch_bounds__(K2_THREADS, 2) verify_kernel(const VerifyParam
         if (lane == 0) s_path[m] = u;
         continue;
       }
+      const double inv = 1.0 / zr;
+      scale = pq * inv;
       nsup = nc;
-      if (lane < nc) { s_sup_id[lane] = cid; s_sup_pt[lane] = pt; s_sup_p[lane] = s_p[u][lane]; }
+      if (lane < nc) { s_sup_id[lane] = cid; s_sup_pt[lane] = ph * inv; s_sup_p[lane] = s_p[u][lane]; }
       break;
     }
     if (lane == 0) {
@@ -335,7 +394,7 @@ __global__ void __launch_bounds__(K2_THREADS, 2) verify_kernel(const VerifyParam
   const int nsup = s_nsup;
   const double scale = s_scale;
   const float off = s_off[us];
-  const double Z = s_Z[us];
+  const double invZ = s_invZ[us];
   const double U = (double)philox_u24(p.seed, b, p.step, us, SLOT_FINAL) * (1.0 / 16777216.0);
 
   // coarse: mass of every chunk; thread t owns `per` consecutive chunks
@@ -348,7 +407,7 @@ __global__ void __launch_bounds__(K2_THREADS, 2) verify_kernel(const VerifyParam
     const int ch = tid * per + i;
     if (i < per && ch < p.n_chunks) {
       const float2 pr = p.pairs[rows * p.n_chunks + ch];
-      double mass = scale * (chunk_mass(pr, p.c, off) / Z);
+      double mass = scale * (chunk_mass(pr, p.c, off) * invZ);
       for (int s = 0; s < nsup; ++s)
         if (s_sup_id[s] / CHUNK == ch) mass += s_sup_pt[s] - scale * s_sup_p[s];
       cm[i] = fmax(mass, 0.0);
@@ -401,7 +460,7 @@ __global__ void __launch_bounds__(K2_THREADS, 2) verify_kernel(const VerifyParam
       if (s_hit >= 0) w[e] = s_sup_pt[s_hit];
       else {
         const float x = load_logit(p.logits, p.dtype, rows * (long long)p.V + v);
-        w[e] = scale * (exp2_d((double)x * cd - (double)off) / Z);
+        w[e] = scale * (exp2_d((double)x * cd - (double)off) * invZ);
       }
     }
     wsum += w[e];
@@ -465,19 +524,7 @@ __global__ void __launch_bounds__(K2_THREADS, 2) verify_kernel(const VerifyParam
     __syncthreads();
     if (warp < nr) {
       const float2* pairs = p.pairs + ((long long)b * N + s_path[j0 + warp]) * p.n_chunks;
-      float tau = -INFINITY;
-      if (p.n_chunks >= K) {
-        unsigned long long below = ~0ull;
-        for (int r = 0; r < K; ++r) {
-          unsigned long long best = 0ull;
-          for (int ch = lane; ch < p.n_chunks; ch += 32) {
-            const unsigned long long key = select_key(__float_as_uint(pairs[ch].y), (uint32_t)ch);
-            if (key < below && key > best) best = key;
-          }
-          below = warp_max_u64(best);
-        }
-        tau = key_value(below);
-      }
+      const float tau = kth_largest_chunk_max(pairs, p.n_chunks, K, lane);
       if (lane == 0) s_floor[warp] = tau;
       for (int ch = lane; ch < p.n_chunks; ch += 32)
         if (pairs[ch].y >= tau) {
@@ -511,21 +558,25 @@ __global__ void __launch_bounds__(K2_THREADS, 2) verify_kernel(const VerifyParam
         // selection copes with any input, one chunk at a time
         n = row_topk_warp(p.logits, p.dtype, row, p.V, p.pairs + row * p.n_chunks, p.n_chunks, K, s_cand[warp],
                           &s_ncand[warp], lane);
-      } else {
-        if (n > 0) compact_topk(s_cand[warp], &s_ncand[warp], n, K, lane, s_floor[warp]);
+      } else if (n > 32) {
+        compact_topk(s_cand[warp], &s_ncand[warp], n, K, lane, s_floor[warp]);
         n = n < K ? n : K;
       }
-      if (lane < K) {
-        const long long at = ((long long)b * W1 + j) * K + lane;
-        if (lane < n) {
-          const uint2 e = s_cand[warp][lane];
-          p.rec_ids[at] = (int)e.y;
-          p.rec_p[at] = (float)(exp2_d((double)__uint_as_float(e.x) * cd - (double)s_off[u]) / s_Z[u]);
-        } else {
-          p.rec_ids[at] = -1;
-          p.rec_p[at] = 0.0f;
-        }
+      // one candidate per lane: its rank among them decides its place in the record
+      const uint2 e = lane < n ? s_cand[warp][lane] : make_uint2(0u, 0u);
+      unsigned long long cur = lane < n ? select_key(e.x, e.y) : 0ull;
+      int rank = -1;
+      const int keep = n < K ? n : K;
+      for (int r = 0; r < keep; ++r) {
+        const unsigned long long mx = warp_max_u64(cur);
+        if (cur == mx && cur != 0ull) { rank = r; cur = 0ull; }  // ids are distinct, so are the keys
       }
+      const long long at0 = ((long long)b * W1 + j) * K;
+      if (rank >= 0) {
+        p.rec_ids[at0 + rank] = (int)e.y;
+        p.rec_p[at0 + rank] = (float)(exp2_d((double)__uint_as_float(e.x) * cd - (double)s_off[u]) * s_invZ[u]);
+      }
+      if (lane >= keep && lane < K) { p.rec_ids[at0 + lane] = -1; p.rec_p[at0 + lane] = 0.0f; }
     }
     __syncthreads();
   }
