@@ -45,6 +45,15 @@ __device__ __forceinline__ uint32_t philox_u24(unsigned long long seed, uint32_t
 }
 
 // ---------------------------------------------------------------------------
+// Programmatic dependent launch: a kernel of the step lets the next one start being scheduled at once
+// (pdl_trigger) and the next one stops before it reads anything the previous one wrote (pdl_wait, which
+// returns once the previous grid has completed and its writes are visible).  Both are no-ops in a kernel
+// that was launched without the attribute.
+// ---------------------------------------------------------------------------
+__device__ __forceinline__ void pdl_trigger() { asm volatile("griddepcontrol.launch_dependents;" ::: "memory"); }
+__device__ __forceinline__ void pdl_wait() { asm volatile("griddepcontrol.wait;" ::: "memory"); }
+
+// ---------------------------------------------------------------------------
 // warp helpers
 // ---------------------------------------------------------------------------
 __device__ __forceinline__ float warp_max_f(float v) {

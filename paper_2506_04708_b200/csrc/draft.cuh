@@ -59,6 +59,7 @@ __global__ void __launch_bounds__(K4_THREADS) draft_kernel(const DraftParams p) 
   __shared__ Slot s_slot[K4_THREADS / 32];  // per warp: the slot that won the lookup
   const int b = blockIdx.x, tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
   const int N = p.N, K = p.K, n_max = p.n_max;
+  pdl_trigger();
   // topology and tail once, with coalesced loads: the level loop below touches shared memory only
   for (int u = tid; u < N; u += K4_THREADS) {
     s_tok[u] = -1;
@@ -66,8 +67,9 @@ __global__ void __launch_bounds__(K4_THREADS) draft_kernel(const DraftParams p) 
     s_fc[u] = p.first_child[u];
     s_nch[u] = p.n_children[u];
   }
-  if (tid < n_max) s_tail[tid] = p.tail[b * n_max + tid];
   if (tid <= p.D + 1) s_level[tid] = p.level_start[tid];
+  pdl_wait();  // tails come from the verification, the table from the update
+  if (tid < n_max) s_tail[tid] = p.tail[b * n_max + tid];
   __syncthreads();
   if (tid == 0) s_tok[0] = s_tail[n_max - 1];  // the root carries the last token
   __syncthreads();

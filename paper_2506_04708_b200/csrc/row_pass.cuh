@@ -228,6 +228,7 @@ __global__ void __launch_bounds__((CW + 1) * 32, CTAS) row_pass_kernel(const Row
   __shared__ volatile int s_abort;
 
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  pdl_trigger();  // a dependent kernel may be scheduled as soon as resources free up; it waits for this grid's end
   const long long t0 = (long long)blockIdx.x * p.total_tiles / gridDim.x;
   const long long t1 = (long long)(blockIdx.x + 1) * p.total_tiles / gridDim.x;
   const int n_tiles = (int)(t1 - t0);

@@ -183,6 +183,23 @@ int launch_row_pass(const void* logits, long long rows, int V, int dtype, int n_
   return launch_ok();
 }
 
+// Launch with programmatic stream serialisation: the kernel may be scheduled while its predecessor in the
+// stream is still running; it calls pdl_wait() before it touches the predecessor's results.
+template <typename P>
+int launch_dependent(void (*kernel)(P), unsigned grid, unsigned block, cudaStream_t st, const P& params) {
+  cudaLaunchConfig_t cfg = {};
+  cfg.gridDim = dim3(grid);
+  cfg.blockDim = dim3(block);
+  cfg.dynamicSmemBytes = 0;
+  cfg.stream = st;
+  cudaLaunchAttribute attr[1];
+  attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+  attr[0].val.programmaticStreamSerializationAllowed = 1;
+  cfg.attrs = attr;
+  cfg.numAttrs = 1;
+  return cuda_ok(cudaLaunchKernelEx(&cfg, kernel, params));
+}
+
 UpdateParams update_params(stand_ctx* x, long long n_rows, const int* ctxw, const int* ids, const float* probs,
                            const int* n_path, int width) {
   const stand_config& c = x->cfg;
@@ -224,8 +241,10 @@ int run_verify(stand_ctx* x, const void* logits, int32_t* emitted, int32_t* n_em
   v.stats = x->at<unsigned long long>(x->L.stats);
   v.fuse_locate = fuse_locate ? 1 : 0;
   v.upd = step_update_params(x);
-  verify_kernel<<<c.B, K2_THREADS, 0, st>>>(v);
-  rc = launch_ok();
+  // inside a fused step (and with no timing events between the launches) the kernels chain programmatically
+  const bool chain = fuse_locate && !x->ev_after && !x->ev_stage[1];
+  if (chain) rc = launch_dependent(verify_kernel, (unsigned)c.B, K2_THREADS, st, v);
+  else { verify_kernel<<<c.B, K2_THREADS, 0, st>>>(v); rc = launch_ok(); }
   if (rc) return rc;
   if (x->ev_stage[2]) cudaEventRecord(x->ev_stage[2], st);
   x->launches += 1;
@@ -243,8 +262,9 @@ int run_update_rows(stand_ctx* x, const UpdateParams& u, bool located, cudaStrea
     if (rc) return rc;
     x->launches += 1;
   }
-  update_apply_kernel<<<(unsigned)((n_rec + APPLY_WARPS - 1) / APPLY_WARPS), APPLY_WARPS * 32, 0, st>>>(u);
-  rc = launch_ok();
+  const unsigned apply_blocks = (unsigned)((n_rec + APPLY_WARPS - 1) / APPLY_WARPS);
+  if (located && !x->ev_stage[2]) rc = launch_dependent(update_apply_kernel, apply_blocks, APPLY_WARPS * 32, st, u);
+  else { update_apply_kernel<<<apply_blocks, APPLY_WARPS * 32, 0, st>>>(u); rc = launch_ok(); }
   if (rc) return rc;
   x->launches += 1;
   return STAND_OK;
@@ -257,7 +277,7 @@ int run_update(stand_ctx* x, cudaStream_t st) {
   return rc;
 }
 
-int run_draft(stand_ctx* x, int32_t* tree_user, cudaStream_t st) {
+int run_draft(stand_ctx* x, int32_t* tree_user, bool chained, cudaStream_t st) {
   const stand_config& c = x->cfg;
   DraftParams d;
   d.table = x->at<Slot>(x->L.table); d.mask = c.table_slots - 1; d.max_probe = x->max_probe; d.B = c.B; d.N = c.N;
@@ -266,8 +286,9 @@ int run_draft(stand_ctx* x, int32_t* tree_user, cudaStream_t st) {
   d.level_start = x->topo_level_start(); d.tail = x->at<int>(x->L.tail); d.tree = x->at<int>(x->L.tree);
   d.tree_user = tree_user; d.cand_n = x->at<int>(x->L.cand_n); d.cand_id = x->at<int>(x->L.cand_id);
   d.cand_phi = x->at<float>(x->L.cand_phi); d.stats = x->at<unsigned long long>(x->L.stats);
-  draft_kernel<<<c.B, K4_THREADS, 0, st>>>(d);
-  const int rc = launch_ok();
+  int rc;
+  if (chained && !x->ev_stage[3]) rc = launch_dependent(draft_kernel, (unsigned)c.B, K4_THREADS, st, d);
+  else { draft_kernel<<<c.B, K4_THREADS, 0, st>>>(d); rc = launch_ok(); }
   if (rc == STAND_OK) x->launches += 1;
   if (x->ev_stage[4]) cudaEventRecord(x->ev_stage[4], st);
   return rc;
@@ -401,7 +422,7 @@ int stand_ngram_update_bulk(stand_ctx* x, const int32_t* dev_ctx, const int32_t*
 int stand_draft_tree(stand_ctx* x, int32_t* dev_tree_tokens, void* cu_stream) {
   if (!x) return STAND_E_ARG;
   x->last_stream = (cudaStream_t)cu_stream;
-  return run_draft(x, dev_tree_tokens, (cudaStream_t)cu_stream);
+  return run_draft(x, dev_tree_tokens, false, (cudaStream_t)cu_stream);
 }
 
 int stand_step(stand_ctx* x, const void* dev_logits, int32_t* dev_emitted, int32_t* dev_n_emitted, int32_t* dev_tree_tokens,
@@ -414,7 +435,7 @@ int stand_step(stand_ctx* x, const void* dev_logits, int32_t* dev_emitted, int32
   if (rc) return rc;
   rc = run_update(x, st);
   if (rc) return rc;
-  return run_draft(x, dev_tree_tokens, st);
+  return run_draft(x, dev_tree_tokens, true, st);
 }
 
 int stand_step_host(stand_ctx* x, const void* host_logits, int32_t* host_emitted, int32_t* host_n_emitted,
@@ -431,7 +452,7 @@ int stand_step_host(stand_ctx* x, const void* host_logits, int32_t* host_emitted
   if (rc) return rc;
   rc = run_update(x, st);
   if (rc) return rc;
-  rc = run_draft(x, nullptr, st);
+  rc = run_draft(x, nullptr, true, st);
   if (rc) return rc;
   const size_t W = x->d.D + 1;
   if (host_emitted) rc = cuda_ok(cudaMemcpyAsync(host_emitted, x->ws + x->L.emitted, c.B * W * 4, cudaMemcpyDeviceToHost, st));

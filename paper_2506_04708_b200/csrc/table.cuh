@@ -342,6 +342,8 @@ __global__ void __launch_bounds__(APPLY_WARPS * 32) update_apply_kernel(const Up
   __shared__ SlotImage s_img[APPLY_WARPS];
   const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
   const long long g = (long long)blockIdx.x * APPLY_WARPS + warp;
+  pdl_trigger();
+  pdl_wait();  // records and slot marks come from stage 1
   if (g >= p.n_rows * p.n_max) return;
   // order-major, so that the warps of a block work on neighbouring rows of one order
   const int n = (int)(g / p.n_rows) + 1;

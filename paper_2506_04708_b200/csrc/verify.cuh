@@ -259,7 +259,8 @@ __global__ void __launch_bounds__(K2_THREADS, 2) verify_kernel(const VerifyParam
   const int N = p.N, K = p.K;
   const double cd = (double)p.c;
 
-  // ---- phase 0: stage the sequence's state ------------------------------------------
+  pdl_trigger();
+  // ---- phase 0: stage the sequence's state (written before the row pass of this step began) ------------------------------------------
   for (int u = tid; u < N; u += K2_THREADS) {
     s_tree[u] = p.tree[(long long)b * N + u];
     s_cn[u] = p.cand_n[(long long)b * N + u];
@@ -285,6 +286,7 @@ __global__ void __launch_bounds__(K2_THREADS, 2) verify_kernel(const VerifyParam
     gx[k] = 0.0f;
     if (u < N && t < s_cn[u]) gx[k] = load_logit(p.logits, p.dtype, ((long long)b * N + u) * (long long)p.V + s_cid[u][t]);
   }
+  pdl_wait();  // the chunk pairs come from the row pass
   {
     const int gl = tid & (ROW_LANES - 1);
     for (int u0 = 0; u0 < N; u0 += K2_THREADS / ROW_LANES) {
