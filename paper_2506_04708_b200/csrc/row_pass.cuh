@@ -241,6 +241,7 @@ __global__ void __launch_bounds__((CW + 1) * 32, CTAS) row_pass_kernel(const Row
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
   }
   __syncthreads();
+  pdl_wait();  // chained after the previous step: nothing is read or written before that step has ended
   const size_t row_bytes = (size_t)p.V * TR::ESIZE;
   // tile coordinates advance without divisions
   long long row = t0 / p.tiles_per_row;

@@ -132,6 +132,9 @@ bool rows_aligned(const void* base, int V, int dtype) {
   return ((uintptr_t)base % 16 == 0) && (((size_t)V * es) % 16 == 0);
 }
 
+template <typename P>
+int launch_dependent(void (*kernel)(P), unsigned grid, unsigned block, cudaStream_t st, const P& params, size_t smem = 0);
+
 // The streaming kernel needs more dynamic shared memory than the default limit: raise it once per device.
 constexpr int MAX_DEVICES = 64;
 std::atomic<int> g_k1_ready[MAX_DEVICES];
@@ -158,7 +161,7 @@ int prepare_device(int* sm_count) {
 }
 
 int launch_row_pass(const void* logits, long long rows, int V, int dtype, int n_chunks, float c, float2* pairs, int* status,
-                    cudaStream_t st) {
+                    cudaStream_t st, bool chain = false) {
   RowPassParams rp;
   rp.logits = logits; rp.rows = rows; rp.V = V; rp.n_chunks = n_chunks; rp.c = c; rp.pairs = pairs; rp.status = status;
   const int tile_chunks = dtype == STAND_DTYPE_BF16 ? K1Shape<1>::CW : K1Shape<0>::CW;
@@ -171,6 +174,13 @@ int launch_row_pass(const void* logits, long long rows, int V, int dtype, int n_
     if (rc) return rc;
     const long long want = (long long)K1_CTAS * sms;  // each CTA walks a contiguous range of tiles
     const unsigned grid = (unsigned)(rp.total_tiles < want ? rp.total_tiles : want);
+    if (chain) {  // may be scheduled while the previous step's last kernel drains; waits for it before any access
+      if (dtype == STAND_DTYPE_BF16)
+        return launch_dependent(row_pass_kernel<1, K1Shape<1>::CW, K1_CTAS>, grid, (K1Shape<1>::CW + 1) * 32, st, rp,
+                                (size_t)k1_smem_bytes<1>());
+      return launch_dependent(row_pass_kernel<0, K1Shape<0>::CW, K1_CTAS>, grid, (K1Shape<0>::CW + 1) * 32, st, rp,
+                              (size_t)k1_smem_bytes<0>());
+    }
     if (dtype == STAND_DTYPE_BF16)
       row_pass_kernel<1, K1Shape<1>::CW, K1_CTAS><<<grid, (K1Shape<1>::CW + 1) * 32, k1_smem_bytes<1>(), st>>>(rp);
     else
@@ -186,11 +196,11 @@ int launch_row_pass(const void* logits, long long rows, int V, int dtype, int n_
 // Launch with programmatic stream serialisation: the kernel may be scheduled while its predecessor in the
 // stream is still running; it calls pdl_wait() before it touches the predecessor's results.
 template <typename P>
-int launch_dependent(void (*kernel)(P), unsigned grid, unsigned block, cudaStream_t st, const P& params) {
+int launch_dependent(void (*kernel)(P), unsigned grid, unsigned block, cudaStream_t st, const P& params, size_t smem) {
   cudaLaunchConfig_t cfg = {};
   cfg.gridDim = dim3(grid);
   cfg.blockDim = dim3(block);
-  cfg.dynamicSmemBytes = 0;
+  cfg.dynamicSmemBytes = smem;
   cfg.stream = st;
   cudaLaunchAttribute attr[1];
   attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
@@ -222,7 +232,7 @@ int run_verify(stand_ctx* x, const void* logits, int32_t* emitted, int32_t* n_em
   if (x->ev_before) cudaEventRecord(x->ev_before, st);
   if (x->ev_stage[0]) cudaEventRecord(x->ev_stage[0], st);
   int rc = launch_row_pass(logits, (long long)c.B * c.N, c.V, c.dtype, x->d.n_chunks, x->c, x->at<float2>(x->L.pairs),
-                           x->at<int>(x->L.status), st);
+                           x->at<int>(x->L.status), st, fuse_locate && !x->ev_before && !x->ev_stage[0]);
   if (rc) return rc;
   if (x->ev_after) cudaEventRecord(x->ev_after, st);
   if (x->ev_stage[1]) cudaEventRecord(x->ev_stage[1], st);
