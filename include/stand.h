@@ -223,6 +223,30 @@ int stand_state_load(stand_ctx* ctx, const int32_t* dev_tail, const int64_t* dev
  * after it, so the caller can time that kernel alone.  NULL, NULL switches the hook off. */
 int stand_profile_row_pass(stand_ctx* ctx, void* ev_before, void* ev_after);
 
+/* Sec. 4.2 "Data-driven draft tree optimization", the measuring half: how often each node of the static
+ * tree lay on the accepted path since stand_init (or the last reset).  Synchronises the stream the context
+ * last used, copies N counters to host_counts and, if reset != 0, clears them.  The root is on every path,
+ * so host_counts[0] = sequences x steps. */
+int stand_node_accepts(stand_ctx* ctx, uint64_t* host_counts, int32_t reset);
+
+/* The selecting half: keeps the `keep` nodes with the highest counts (equal counts: the lower index), the
+ * root included.  A node is never accepted more often than its parent, so the kept set is closed under
+ * parents.  Host only.  Writes the parent array of the smaller tree to host_parent_out [keep], in the same
+ * breadth-first numbering convention, and to host_old_index [keep] (may be NULL) the node each kept node
+ * was.  STAND_E_ARG if keep < 1, keep > n or the input is not a valid tree. */
+int stand_prune_tree(const int32_t* host_parent, int32_t n, const uint64_t* host_counts, int32_t keep,
+                     int32_t* host_parent_out, int32_t* host_old_index);
+
+/* App. A.1, Algorithm 1: the initial tree that the optimisation starts from.  Nodes are created level by
+ * level for `levels` levels below the root (20 in the paper: 625 nodes); a node of depth 0 gets 8 children,
+ * of depth 1 max(8 - 2 * order, 1), deeper ones max(ceil((siblings - 1) / (0.7 * order + 1)), floor) with
+ * floor 2 at depths 2 and 3 and 0 below, where `order` is the node's rank among its siblings and
+ * `siblings` its parent's child count; the first node of every level gets at least 3.  Host only.  Writes
+ * the first min(capacity, total) nodes in creation order (a prefix is closed under parents) to
+ * host_parent / host_depth / host_order (the last two may be NULL) and the total to *total_nodes. */
+int stand_initial_tree(int32_t levels, int32_t* host_parent, int32_t* host_depth, int32_t* host_order, int32_t capacity,
+                       int32_t* total_nodes);
+
 /* Timing hook for benchmarks: events [5] (cudaEvent_t as void*, any may be NULL) are recorded on the
  * stream by every later step at: before the row pass, after it, after the verification walk, after the
  * table update, after drafting.  A NULL array switches the hook off. */

@@ -20,7 +20,8 @@ EXPORTS = [
     "stand_ngram_update", "stand_ngram_update_bulk", "stand_draft_tree", "stand_step", "stand_step_host",
     "stand_row_stats_scratch_bytes", "stand_row_stats", "stand_row_stats_static", "stand_get_stats",
     "stand_last_path", "stand_tree_depth", "stand_table_dump", "stand_table_load", "stand_state_dump",
-    "stand_state_load", "stand_profile_row_pass", "stand_profile_stages", "stand_launch_count", "stand_strerror",
+    "stand_state_load", "stand_profile_row_pass", "stand_profile_stages", "stand_node_accepts", "stand_prune_tree",
+    "stand_initial_tree", "stand_launch_count", "stand_strerror",
 ]
 
 
@@ -86,6 +87,12 @@ def lib():
     L.stand_profile_row_pass.restype = C.c_int
     L.stand_profile_stages.argtypes = [vp, C.POINTER(vp)]
     L.stand_profile_stages.restype = C.c_int
+    L.stand_node_accepts.argtypes = [vp, vp, i32]
+    L.stand_node_accepts.restype = C.c_int
+    L.stand_prune_tree.argtypes = [vp, i32, vp, i32, vp, vp]
+    L.stand_prune_tree.restype = C.c_int
+    L.stand_initial_tree.argtypes = [i32, vp, vp, vp, i32, C.POINTER(i32)]
+    L.stand_initial_tree.restype = C.c_int
     L.stand_launch_count.argtypes = [vp]
     L.stand_launch_count.restype = u64
     L.stand_strerror.argtypes = [C.c_int]
@@ -245,6 +252,12 @@ class Stand:
         arr = (C.c_void_p * 5)(*[C.c_void_p(e.cuda_event) for e in events])
         _check(lib().stand_profile_stages(self.h, arr), "stand_profile_stages")
 
+    def node_accepts(self, reset=False):
+        """How often each tree node lay on the accepted path (numpy uint64 [N])."""
+        out = np.zeros(self.N, np.uint64)
+        _check(lib().stand_node_accepts(self.h, out.ctypes.data, int(reset)), "stand_node_accepts")
+        return out
+
     def lens_device(self, out):
         """Copies the sequence lengths into `out` (int64 [B], device) on the current stream."""
         _check(lib().stand_state_dump(self.h, None, _ptr(out), None, None, None, None, None, _stream(None)),
@@ -368,3 +381,24 @@ def row_stats_static(logits, temperature, topk, out=None, stream=None):
                                             _ptr(vals), _ptr(probs), _stream(stream)), "stand_row_stats_static")
     (torch.cuda.current_stream() if stream is None else stream).synchronize()
     return out
+
+
+def initial_tree(levels=20, capacity=None):
+    """App. A.1 Algorithm 1: (parent, depth, order, total_nodes); at most `capacity` nodes are returned."""
+    total = C.c_int32()
+    _check(lib().stand_initial_tree(levels, None, None, None, 0, C.byref(total)), "stand_initial_tree")
+    n = total.value if capacity is None else min(capacity, total.value)
+    parent, depth, order = (np.zeros(n, np.int32) for _ in range(3))
+    _check(lib().stand_initial_tree(levels, parent.ctypes.data, depth.ctypes.data, order.ctypes.data, n, C.byref(total)),
+           "stand_initial_tree")
+    return parent, depth, order, total.value
+
+
+def prune_tree(parent, counts, keep):
+    """Keeps the `keep` most often accepted nodes: (new parent array, old index of every kept node)."""
+    par = np.ascontiguousarray(parent, np.int32)
+    cnt = np.ascontiguousarray(counts, np.uint64)
+    out, old = np.zeros(keep, np.int32), np.zeros(keep, np.int32)
+    _check(lib().stand_prune_tree(par.ctypes.data, len(par), cnt.ctypes.data, keep, out.ctypes.data, old.ctypes.data),
+           "stand_prune_tree")
+    return out, old

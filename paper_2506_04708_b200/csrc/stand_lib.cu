@@ -5,6 +5,7 @@
 #include <cuda_runtime.h>
 #include <atomic>
 #include <new>
+#include <vector>
 #include <stdio.h>
 #include <string.h>
 
@@ -22,7 +23,7 @@ constexpr int BULK_ROWS = 16384;  // rows per batch of the bulk update
 
 struct Layout {
   size_t table, topo, tail, len, tree, cand_n, cand_id, cand_phi, pairs, emitted, n_path, path, rec_ctx, rec_ids,
-      rec_p, rec_slot, stats, status, staging, total;
+      rec_p, rec_slot, stats, accepts, status, staging, total;
 };
 
 inline size_t align_up(size_t x) { return (x + 255) & ~(size_t)255; }
@@ -90,6 +91,7 @@ void layout_of(const stand_config* c, const Derived* d, Layout* L) {
   L->rec_p = take(B * W * K * 4);
   L->rec_slot = take(rec_rows * n * 4);
   L->stats = take(ST_COUNT * 8);
+  L->accepts = take(NODES_MAX * 8);
   L->status = take(64);
   L->staging = take(c->host_staging ? B * N * (size_t)c->V * esize_of(c->dtype) : 0);
   L->total = at;
@@ -249,6 +251,7 @@ int run_verify(stand_ctx* x, const void* logits, int32_t* emitted, int32_t* n_em
   v.emitted = x->at<int>(x->L.emitted); v.n_path = x->at<int>(x->L.n_path); v.path = x->at<int>(x->L.path);
   v.rec_ctx = x->at<int>(x->L.rec_ctx); v.rec_ids = x->at<int>(x->L.rec_ids); v.rec_p = x->at<float>(x->L.rec_p);
   v.stats = x->at<unsigned long long>(x->L.stats);
+  v.node_accepts = x->at<unsigned long long>(x->L.accepts);
   v.fuse_locate = fuse_locate ? 1 : 0;
   v.upd = step_update_params(x);
   // inside a fused step (and with no timing events between the launches) the kernels chain programmatically
@@ -653,6 +656,80 @@ int stand_profile_row_pass(stand_ctx* x, void* ev_before, void* ev_after) {
   if (!x || ((ev_before == nullptr) != (ev_after == nullptr))) return STAND_E_ARG;
   x->ev_before = (cudaEvent_t)ev_before;
   x->ev_after = (cudaEvent_t)ev_after;
+  return STAND_OK;
+}
+
+int stand_node_accepts(stand_ctx* x, uint64_t* host_counts, int32_t reset) {
+  if (!x || !host_counts) return STAND_E_ARG;
+  int rc = cuda_ok(cudaStreamSynchronize(x->last_stream));
+  if (rc) return rc;
+  rc = cuda_ok(cudaMemcpy(host_counts, x->ws + x->L.accepts, (size_t)x->cfg.N * 8, cudaMemcpyDeviceToHost));
+  if (rc == STAND_OK && reset) rc = cuda_ok(cudaMemset(x->ws + x->L.accepts, 0, (size_t)x->cfg.N * 8));
+  return rc;
+}
+
+int stand_prune_tree(const int32_t* host_parent, int32_t n, const uint64_t* host_counts, int32_t keep,
+                     int32_t* host_parent_out, int32_t* host_old_index) {
+  if (!host_parent || !host_counts || !host_parent_out || n < 1 || keep < 1 || keep > n || host_parent[0] != -1) return STAND_E_ARG;
+  for (int32_t u = 1; u < n; ++u)
+    if (host_parent[u] < 0 || host_parent[u] >= u) return STAND_E_ARG;
+  // a node is kept if fewer than `keep` nodes come before it in (count descending, index ascending) order
+  std::vector<char> kept((size_t)n, 0);
+  std::vector<int32_t> new_index((size_t)n, -1);
+  for (int32_t u = 0; u < n; ++u) {
+    int32_t before = 0;
+    for (int32_t w = 0; w < n; ++w)
+      if (host_counts[w] > host_counts[u] || (host_counts[w] == host_counts[u] && w < u)) ++before;
+    kept[u] = before < keep ? 1 : 0;
+  }
+  if (!kept[0]) return STAND_E_ARG;  // the root is on every path: counts that rank it out are not acceptance counts
+  int32_t at = 0;
+  for (int32_t u = 0; u < n; ++u) {  // the old numbering is breadth-first with siblings together: so is the new one
+    if (!kept[u]) continue;
+    if (u > 0 && !kept[host_parent[u]]) return STAND_E_ARG;  // counts that grow towards the leaves: not acceptance counts
+    new_index[u] = at;
+    host_parent_out[at] = u == 0 ? -1 : new_index[host_parent[u]];
+    if (host_old_index) host_old_index[at] = u;
+    ++at;
+  }
+  return at == keep ? STAND_OK : STAND_E_ARG;
+}
+
+int stand_initial_tree(int32_t levels, int32_t* host_parent, int32_t* host_depth, int32_t* host_order, int32_t capacity,
+                       int32_t* total_nodes) {
+  if (levels < 0 || levels > 64 || !total_nodes || capacity < 0 || (capacity > 0 && !host_parent)) return STAND_E_ARG;
+  struct Node { int32_t parent, depth, order, n_children; };
+  std::vector<Node> nodes;
+  nodes.push_back({-1, 0, 0, 0});
+  size_t level_begin = 0, level_end = 1;  // the nodes of the current level are nodes[level_begin, level_end)
+  for (int32_t l = 0; l < levels; ++l) {
+    for (size_t at = level_begin; at < level_end; ++at) {
+      const Node me = nodes[at];
+      int64_t n;
+      if (me.depth == 0) n = 8;
+      else if (me.depth == 1) n = 8 - 2 * me.order > 1 ? 8 - 2 * me.order : 1;
+      else {
+        // ceil((siblings - 1) / (0.7 * order + 1)) in integers: ceil(10 (siblings - 1) / (7 order + 10))
+        const int64_t num = 10 * (int64_t)(nodes[me.parent].n_children - 1), den = 7 * (int64_t)me.order + 10;
+        n = (num + den - 1) / den;
+        const int64_t floor = (me.depth == 2 || me.depth == 3) ? 2 : 0;
+        if (n < floor) n = floor;
+      }
+      if (at == level_begin && n < 3) n = 3;
+      if (nodes.size() + (size_t)n > (1u << 24)) return STAND_E_ARG;
+      nodes[at].n_children = (int32_t)n;
+      for (int32_t k = 0; k < (int32_t)n; ++k) nodes.push_back({(int32_t)at, me.depth + 1, k, 0});
+    }
+    level_begin = level_end;
+    level_end = nodes.size();
+  }
+  *total_nodes = (int32_t)nodes.size();
+  const size_t out = nodes.size() < (size_t)capacity ? nodes.size() : (size_t)capacity;
+  for (size_t i = 0; i < out; ++i) {
+    host_parent[i] = nodes[i].parent;
+    if (host_depth) host_depth[i] = nodes[i].depth;
+    if (host_order) host_order[i] = nodes[i].order;
+  }
   return STAND_OK;
 }
 

@@ -51,6 +51,7 @@ struct VerifyParams {
   int* rec_ids;            // [B, D+1, K]
   float* rec_p;            // [B, D+1, K]
   unsigned long long* stats;
+  unsigned long long* node_accepts;  // [N] how often each node lay on an accepted path
   int fuse_locate;         // != 0: also run stage 1 of the N-gram update for this sequence's records
   UpdateParams upd;        // used when fuse_locate is set
 };
@@ -511,6 +512,7 @@ __global__ void __launch_bounds__(K2_THREADS, 2) verify_kernel(const VerifyParam
     p.emitted[b * W1 + tid] = e;
     if (p.emitted_user) p.emitted_user[b * W1 + tid] = e;
     p.path[b * W1 + tid] = tid <= m ? s_path[tid] : -1;
+    if (tid <= m) atomicAdd(&p.node_accepts[s_path[tid]], 1ull);
   }
   // Compressed rows of the accepted path: the exact top-k of each row, as probabilities.  The k-th
   // largest chunk maximum bounds the k-th largest entry from below, so only the chunks whose maximum

@@ -68,10 +68,10 @@ class ClosedLoop:
     """Runs the same seeded workload through both sides, step by step."""
 
     def __init__(self, w, seed=0, peak_mode="add8", table_slots=None, prompt=8, device="cuda:0", device_logits=False,
-                 **stand_kw):
+                 parent=None, **stand_kw):
         from paper_2506_04708_b200.binding import Stand
         self.w, self.seed, self.peak_mode = w, seed, peak_mode
-        self.parent = inputs.topology(w.N, w.D, w.kb)
+        self.parent = inputs.topology(w.N, w.D, w.kb) if parent is None else np.ascontiguousarray(parent, np.int32)
         self.depth = inputs.node_depths(self.parent)
         self.streams = inputs.token_streams(w, seed, prompt + (w.steps + 2) * (w.D + 2))
         slots = table_slots or w.table_slots

@@ -132,6 +132,45 @@ def test_tiny_shapes(V, N, D, kb, dtype):
     _run(w, 60, "p80", check_every=20)
 
 
+# ------------------------------------------------ acceptance counters and tree optimisation (Sec. 4.2)
+def test_node_acceptance_counters_and_tree_optimisation():
+    """Data-driven tree optimisation on a synthetic workload: start from (a 128-node prefix of) Algorithm 1's
+    tree, count how often each node is accepted, keep the most accepted nodes, run on with the smaller tree."""
+    from paper_2506_04708_b200 import binding
+    parent, depth, _, total = binding.initial_tree(20, capacity=128)
+    assert total == 625
+    D = int(depth.max())
+    w = inputs.Workload("opt", 6, 128, D, 8, 3000, inputs.DTYPE_F32, 0.9, 3, 8, 50, 1 << 14, 2.0, 0.7, 16, 1.1)
+    loop = harness.ClosedLoop(w, seed=2, peak_mode="p80", parent=parent)
+    counts = np.zeros(128, np.uint64)
+    try:
+        for _ in range(w.steps):
+            loop.step()
+            for row in loop.orc.path():
+                for u in row[row >= 0]:
+                    counts[u] += 1
+        assert loop.hard == [] and loop.tolerated <= 2
+        got = loop.gpu.node_accepts()
+        if loop.tolerated == 0:
+            assert np.array_equal(got, counts)
+        assert got[0] == w.B * w.steps and got[1:].sum() > 0
+        assert all(got[u] <= got[parent[u]] for u in range(1, 128))
+        small, old = binding.prune_tree(parent, got, 24)
+        assert loop.gpu.node_accepts(reset=True)[0] == got[0] and loop.gpu.node_accepts().sum() == 0
+    finally:
+        loop.close()
+    # the optimised tree is a valid topology and runs in parity too
+    d2 = int(inputs.node_depths(small).max())
+    w2 = inputs.Workload("opt24", 6, 24, d2, 8, 3000, inputs.DTYPE_F32, 0.9, 3, 8, 30, 1 << 14, 2.0, 0.7, 16, 1.1)
+    loop2 = harness.ClosedLoop(w2, seed=2, peak_mode="p80", parent=small)
+    try:
+        for _ in range(w2.steps):
+            loop2.step()
+        assert loop2.hard == [] and loop2.check_state_and_table() == []
+    finally:
+        loop2.close()
+
+
 # ------------------------------------------------------------------- stages on their own
 def test_stage_calls_equal_the_fused_step():
     torch = _torch()
