@@ -17,6 +17,8 @@
 //               static tree asks for without replacement; Gumbel-Top-K:
 //               phi' = phi - log(-log U), keep the largest.
 //   * Sec. 5    sampling temperature T (softmax of logits / T).
+//   * Sec. 3.2  deterministic drafting as a variant: the drafts of a node are
+//               its most probable candidates, each verified as a one-hot draft.
 //
 // Readings where the paper is silent (multi-draft verification by recursive
 // rejection, what q is, inverse-CDF order, canonical update order, ...) are
@@ -210,6 +212,57 @@ int verify_children(const std::vector<double>& p, const std::vector<int>& cand_i
 }
 
 // ---------------------------------------------------------------------------
+// Sec. 3.2, deterministic drafting: the draft distribution of a drafted token x
+// is the one-hot vector at x, so x is accepted with probability pt(x); on
+// rejection the target becomes norm(max(0, pt - onehot(x))), i.e. x loses its
+// mass and the rest is renormalised, and the next child is tested against that.
+// Same arguments and results as verify_children (the candidate list plays no
+// part: the drafts are not sampled).
+// ---------------------------------------------------------------------------
+int verify_children_deterministic(const std::vector<double>& p, const std::vector<int>& child,
+                                  const std::vector<double>& u_acc, double u_final, int* resampled,
+                                  std::vector<double>* accept_margins, double* final_margin) {
+  const int V = (int)p.size();
+  std::vector<double> pt(p);
+  for (size_t j = 0; j < child.size(); ++j) {
+    const int x = child[j];
+    std::vector<double> q(V, 0.0);
+    q[x] = 1.0;
+    const bool accept = u_acc[j] * q[x] < pt[x];
+    if (accept_margins) accept_margins->push_back(std::fabs(u_acc[j] - pt[x] / q[x]));
+    if (accept) return (int)j;
+    double rsum = 0.0;
+    for (int v = 0; v < V; ++v) {
+      pt[v] = std::max(0.0, pt[v] - q[v]);
+      rsum += pt[v];
+    }
+    for (int v = 0; v < V; ++v) pt[v] /= rsum;
+  }
+  *resampled = inverse_cdf(pt, u_final, final_margin);
+  return -1;
+}
+
+// Deterministic drafting: the m most probable candidates, most probable first
+// (equal probabilities: lower token id first).  Returns indices into the list.
+std::vector<int> most_probable(const std::vector<int>& id, const std::vector<double>& phi, int m, double* margin) {
+  const int n = (int)id.size();
+  std::vector<int> order(n);
+  for (int i = 0; i < n; ++i) order[i] = i;
+  std::sort(order.begin(), order.end(), [&](int a, int b) {
+    if (phi[a] != phi[b]) return phi[a] > phi[b];
+    return id[a] < id[b];
+  });
+  const int take = std::min(m, n);
+  if (margin) {
+    double gap = INFINITY;
+    for (int r = 0; r < take && r + 1 < n; ++r) gap = std::min(gap, (phi[order[r]] - phi[order[r + 1]]) / phi[order[r]]);
+    *margin = gap;
+  }
+  order.resize(take);
+  return order;
+}
+
+// ---------------------------------------------------------------------------
 // Sec. 4.2 Gumbel-Top-K: g_i = log phi_i - log(-log U_i); the m largest, in
 // decreasing order (equal g: lower token id first).  Returns indices into the
 // candidate list.
@@ -276,6 +329,7 @@ void merge_entry(Entry& e, const std::vector<std::pair<int, double>>& fresh, int
 // ---------------------------------------------------------------------------
 struct Oracle {
   int B, N, V, K, n_max, dtype;
+  int deterministic = 0;  // 1: deterministic drafting (Sec. 3.2), 0: stochastic (Sec. 4.2)
   double T;
   uint64_t seed;
   std::vector<int> parent, depth;
@@ -340,8 +394,10 @@ struct Oracle {
       int resampled = -1;
       std::vector<double> am;
       double fm = 1.0;
-      const int acc = verify_children(P[u], cand_id[b][u], cand_phi[b][u], drafted_tokens, u_acc,
-                                      u_final, &resampled, &am, &fm);
+      const int acc = deterministic
+                          ? verify_children_deterministic(P[u], drafted_tokens, u_acc, u_final, &resampled, &am, &fm)
+                          : verify_children(P[u], cand_id[b][u], cand_phi[b][u], drafted_tokens, u_acc, u_final,
+                                            &resampled, &am, &fm);
       for (size_t j = 0; j < am.size(); ++j) {
         mr.kind = MARGIN_ACCEPT; mr.aux = (int)j; mr.margin = am[j]; local.push_back(mr);
       }
@@ -438,7 +494,7 @@ struct Oracle {
           U.push_back(uniform_open(random_u24(seed, b, step, u, SLOT_GUMBEL | (uint32_t)it.first)));
         }
       double mg;
-      std::vector<int> chosen = gumbel_top(ids, phis, U, m, &mg);
+      std::vector<int> chosen = deterministic ? most_probable(ids, phis, m, &mg) : gumbel_top(ids, phis, U, m, &mg);
       if (!chosen.empty()) add_margin(MARGIN_GUMBEL, b, u, (int)chosen.size(), nullptr, mg);
       for (size_t r = 0; r < chosen.size(); ++r) tree[b][children[u][r]] = ids[chosen[r]];
       cand_id[b][u] = ids;
@@ -497,6 +553,26 @@ int so_verify_children(const double* p, int V, const int32_t* cand_id, const dou
   return acc;
 }
 
+// Deterministic-drafting verification of the children of one node with explicit uniforms.
+int so_verify_children_deterministic(const double* p, int V, const int32_t* child, int n_child, const double* u_acc,
+                                     double u_final, int32_t* resampled) {
+  std::vector<double> pv(p, p + V), ua(u_acc, u_acc + n_child);
+  std::vector<int> ch(child, child + n_child);
+  int res = -1;
+  const int acc = verify_children_deterministic(pv, ch, ua, u_final, &res, nullptr, nullptr);
+  *resampled = res;
+  return acc;
+}
+
+// The m most probable candidates in order; writes the chosen token ids.
+int so_most_probable(const int32_t* id, const double* phi, int n, int m, int32_t* chosen) {
+  std::vector<int> ids(id, id + n);
+  std::vector<double> ph(phi, phi + n);
+  std::vector<int> c = most_probable(ids, ph, m, nullptr);
+  for (size_t r = 0; r < c.size(); ++r) chosen[r] = ids[c[r]];
+  return (int)c.size();
+}
+
 // Gumbel-Top-K with explicit uniforms in (0,1); writes the chosen token ids.
 int so_gumbel_top(const int32_t* id, const double* phi, const double* U, int n, int m, int32_t* chosen) {
   std::vector<int> ids(id, id + n);
@@ -528,6 +604,7 @@ void* so_create(int B, int N, int V, int topk, int order_max, int dtype, double 
   o->fresh.assign(B, {});
   return o;
 }
+void so_set_deterministic(void* h, int on) { ((Oracle*)h)->deterministic = on ? 1 : 0; }
 void so_destroy(void* h) { delete (Oracle*)h; }
 int so_depth(void* h) { return ((Oracle*)h)->D; }
 

@@ -85,6 +85,24 @@ def verify_children(p, cand_id, cand_phi, child, u_acc, u_final):
     return acc, res.value
 
 
+def verify_children_deterministic(p, child, u_acc, u_final):
+    p = np.ascontiguousarray(p, np.float64)
+    ch = np.ascontiguousarray(child, np.int32)
+    ua = np.ascontiguousarray(u_acc, np.float64)
+    res = C.c_int32(-1)
+    acc = lib().so_verify_children_deterministic(_p(p), len(p), _p(ch), len(ch), _p(ua), C.c_double(u_final),
+                                                 C.byref(res))
+    return acc, res.value
+
+
+def most_probable(ids, phi, m):
+    ids = np.ascontiguousarray(ids, np.int32)
+    phi = np.ascontiguousarray(phi, np.float64)
+    out = np.full(max(m, 1), -1, np.int32)
+    n = lib().so_most_probable(_p(ids), _p(phi), len(ids), m, _p(out))
+    return out[:n]
+
+
 def gumbel_top(ids, phi, U, m):
     ids = np.ascontiguousarray(ids, np.int32)
     phi = np.ascontiguousarray(phi, np.float64)
@@ -98,7 +116,7 @@ MARGIN_ACCEPT, MARGIN_FINAL, MARGIN_GUMBEL, MARGIN_MERGE = 0, 1, 2, 3
 
 
 class Oracle:
-    def __init__(self, B, N, V, topk, order_max, dtype, temperature, seed, parent):
+    def __init__(self, B, N, V, topk, order_max, dtype, temperature, seed, parent, deterministic=False):
         self.B, self.N, self.V, self.K, self.n_max, self.dtype = B, N, V, topk, order_max, dtype
         self.parent = np.ascontiguousarray(parent, np.int32)
         assert len(self.parent) == N
@@ -107,6 +125,8 @@ class Oracle:
         self.h = C.c_void_p(lib().so_create(B, N, V, topk, order_max, dtype, C.c_double(self.T), seed,
                                             _p(self.parent)))
         self.D = lib().so_depth(self.h)
+        if deterministic:
+            lib().so_set_deterministic(self.h, 1)
 
     def close(self):
         if self.h:

@@ -256,6 +256,98 @@ def test_verification_chi_square_through_the_tree_walk():
     assert checked >= 1
 
 
+# --------------------------------------- deterministic drafting (Sec. 3.2), the variant
+def test_deterministic_draft_is_accepted_with_its_target_probability():
+    """Sec. 3.2: with a one-hot draft distribution "the drafted token is accepted with p(x_draft)"."""
+    p = np.array([0.1, 0.2, 0.3, 0.4])
+    for x in range(4):
+        thr = _threshold(lambda U, x=x: so.verify_children_deterministic(p, [x], [U], 0.0)[0] == 0)
+        assert abs(thr / 2.0 ** 24 - p[x]) < 2.0 ** -23
+    # on rejection the resample follows norm(max(0, p - onehot)): x loses its mass
+    r = np.array([0.1, 0.2, 0.0, 0.4]) / 0.7
+    cdf = np.cumsum(r)
+    for U in [0.0, 0.14, 0.15, 0.42, 0.43, 0.999]:
+        acc, y = so.verify_children_deterministic(p, [2], [0.9], U)
+        assert acc == -1 and y == int(np.searchsorted(cdf, U, side="right")) and y != 2
+
+
+@pytest.mark.parametrize("case", range(3))
+def test_deterministic_verification_is_lossless_exactly(case):
+    """Several deterministic drafts tested one after the other: the output still follows p exactly.  The oracle is
+    used as a black box (thresholds by bisection over the 24-bit uniforms)."""
+    rng = np.random.default_rng(200 + case)
+    V = [5, 9, 14][case]
+    m = [1, 3, 4][case]
+    p = rng.random(V) ** 2
+    p /= p.sum()
+    child = list(rng.choice(V, m, replace=False))
+    out = np.zeros(V)
+    reach = 1.0
+    for j in range(m):
+        def accepted_j(U, j=j):
+            ua = [1 - 2.0 ** -24] * m
+            ua[j] = U
+            return so.verify_children_deterministic(p, child[:j + 1], ua[:j + 1], 0.0)[0] == j
+        a_j = _threshold(accepted_j) / 2.0 ** 24
+        out[child[j]] += reach * a_j
+        reach *= 1 - a_j
+    ua = [1 - 2.0 ** -24] * m
+    prev = 0
+    for v in range(V):
+        hi = _threshold(lambda U, v=v: so.verify_children_deterministic(p, child, ua, U)[1] <= v, lo=prev)
+        out[v] += reach * (hi - prev) / 2.0 ** 24
+        prev = hi
+    assert np.abs(out - p).max() < 2e-6, (out, p)
+
+
+def test_deterministic_drafts_are_the_most_probable_candidates():
+    ids = np.array([40, 7, 19, 3, 28])
+    phi = np.array([0.1, 0.3, 0.3, 0.05, 0.2])
+    assert list(so.most_probable(ids, phi, 3)) == [7, 19, 28]      # equal probabilities: lower id first
+    assert list(so.most_probable(ids, phi, 9)) == [7, 19, 28, 40, 3]
+    # through the whole oracle: the tree holds the top candidates in order and no randomness enters drafting
+    parent = np.array([-1, 0, 0, 0], np.int32)
+    trees = []
+    for seed in (1, 2):
+        o = so.Oracle(1, 4, 50, 5, 2, 0, 1.0, seed, parent, deterministic=True)
+        i = np.array([[40, 7, 19, 3, 28]], np.int32)
+        o.update_bulk(np.array([[-1, 9]], np.int32), i, phi[None].astype(np.float32))
+        o.reset_sequences(np.array([[-1, 9]], np.int32), np.array([1]))
+        trees.append(o.draft()[0].tolist())
+        o.close()
+    assert trees[0] == trees[1] == [9, 7, 19, 28]
+
+
+def test_deterministic_walk_chi_square():
+    """1e5 trials through the full oracle in deterministic mode (table -> top candidates -> tree verification):
+    the first emitted token follows the root's target distribution."""
+    V, K = 12, 4
+    parent = np.array([-1, 0, 0, 0, 1, 1, 2], np.int32)
+    N = len(parent)
+    rng = np.random.default_rng(6)
+    logits = (rng.standard_normal((1, N, V)) * 1.5).astype(np.float32)
+    T, Bn, reps = 0.8, 250, 400
+    big = np.ascontiguousarray(np.broadcast_to(logits, (Bn, N, V)))
+    first = np.zeros(V)
+    accepted = 0
+    for rep in range(reps):
+        o = so.Oracle(Bn, N, V, K, 2, 0, T, 5000 + rep, parent, deterministic=True)
+        ctx = np.array([[-1, t] for t in range(V)], np.int32)
+        ids = np.array([[(t + 1 + 2 * i) % V for i in range(K)] for t in range(V)], np.int32)
+        probs = np.tile(np.array([0.5, 0.2, 0.2, 0.1], np.float32), (V, 1))
+        o.update_bulk(ctx, ids, probs)
+        o.reset_sequences(np.tile(np.array([-1, 3], np.int32), (Bn, 1)), np.full(Bn, 1))
+        tree = o.draft()
+        assert (tree == tree[0]).all()  # no randomness in deterministic drafting
+        em, ne = o.verify(big)
+        np.add.at(first, em[:, 0], 1)
+        accepted += int((ne >= 2).sum())
+        o.close()
+    _, _, _, _, p0 = so.row_stats(logits[0, 0], float(np.float32(T)), K, want_p=True)
+    assert accepted > 0
+    assert stats.chisquare(first, p0 * first.sum()).pvalue > 0.01
+
+
 # ------------------------------------------------------ N-gram module (Sec. 4.1)
 def test_merge_hand_cases():
     for line in open(os.path.join(GOLD, "merge_cases.txt")):
