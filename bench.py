@@ -198,7 +198,7 @@ def run_ours(args, rank, world, local):
         ring_n = args.ring
 
     gpu = Stand(w.B, w.N, w.V, w.topk, w.order_max, w.dtype, w.T, seed, w.table_slots, parent, device=dev,
-                host_staging=True)
+                host_staging=True, deterministic=args.deterministic)
     contexts = pregrow(gpu, w, seed, torch)
     prompt = 8
     streams = inputs.token_streams(w, seed, prompt + (ring_n + 4) * (w.D + 2))
@@ -329,6 +329,7 @@ def run_ours(args, rank, world, local):
             "warmup": max(args.warmup, 3) + ring_n, "ms_per_step": ms_per_step, "higher_is_better": True,
             "scaling": "weak", "vs_baseline": None, "dtype": "f32", "data": "synthetic",
             "config": {"workload": describe(w), "peak_mode": args.peak_mode, "ring_buffers": ring_n,
+                       "drafting": "deterministic" if args.deterministic else "stochastic (Gumbel-Top-K)",
                        "l2": f"inputs larger than L2: {step_bytes / 1e6:.0f} MB per step, ring of {ring_n} "
                              f"buffers = {ring_n * step_bytes / 1e9:.2f} GB",
                        "table_contexts_at_start": int(contexts), "multi_gpu": "independent replicas per GPU"
@@ -421,6 +422,7 @@ def main():
     ap.add_argument("--peak-mode", default="add8", choices=["add8", "p80"])
     ap.add_argument("--seed", type=int, default=0)
     ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--deterministic", action="store_true", help="deterministic drafting (paper Sec. 3.2) instead of stochastic")
     ap.add_argument("--no-sweep", action="store_true", help="skip the short runs of the other four workloads")
     ap.add_argument("--batch", type=int, default=0, help="override the workload's number of sequences (profiling)")
     ap.add_argument("--ring", type=int, default=0, help="override the number of logit buffers in the ring (profiling)")

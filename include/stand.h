@@ -68,7 +68,8 @@ typedef struct {
   uint64_t seed;
   uint64_t table_slots;   /* power of two, >= 2; one slot = 128 bytes */
   const int32_t* parent;  /* HOST, [N]; parent[0] = -1; read during stand_init only */
-  int32_t reserved;        /* must be 0 */
+  int32_t deterministic;   /* 0: stochastic drafting (Sec. 4.2); 1: deterministic drafting (Sec. 3.2): the children of a
+                              node are its most probable candidates in order, each verified as a one-hot draft */
   int32_t host_staging;    /* != 0: reserve a logits staging buffer for stand_step_host */
 } stand_config;
 

@@ -29,7 +29,7 @@ class StandConfig(C.Structure):
     _fields_ = [
         ("B", C.c_int32), ("N", C.c_int32), ("V", C.c_int32), ("topk", C.c_int32), ("order_max", C.c_int32),
         ("dtype", C.c_int32), ("temperature", C.c_float), ("max_probe", C.c_int32), ("seed", C.c_uint64),
-        ("table_slots", C.c_uint64), ("parent", C.c_void_p), ("reserved", C.c_int32),
+        ("table_slots", C.c_uint64), ("parent", C.c_void_p), ("deterministic", C.c_int32),
         ("host_staging", C.c_int32),
     ]
 
@@ -122,10 +122,10 @@ def _stream(stream):
 
 
 def make_config(B, N, V, topk, order_max, dtype, temperature, seed, table_slots, parent, max_probe=0,
-                host_staging=False):
+                host_staging=False, deterministic=False):
     par = np.ascontiguousarray(parent, np.int32)
     cfg = StandConfig(B, N, V, topk, order_max, dtype, float(temperature), max_probe, seed, table_slots,
-                      par.ctypes.data, 0, int(bool(host_staging)))
+                      par.ctypes.data, int(bool(deterministic)), int(bool(host_staging)))
     cfg._keepalive = par
     return cfg
 
@@ -138,13 +138,13 @@ class Stand:
     """One decoder context.  Tensors are torch CUDA tensors; results are written in place."""
 
     def __init__(self, B, N, V, topk, order_max, dtype, temperature, seed, table_slots, parent, max_probe=0,
-                 host_staging=False, device="cuda:0"):
+                 host_staging=False, device="cuda:0", deterministic=False):
         import torch
         self.torch = torch
         self.dev = torch.device(device)
         self.B, self.N, self.V, self.K, self.n_max, self.dtype = B, N, V, topk, order_max, dtype
         self.cfg = make_config(B, N, V, topk, order_max, dtype, temperature, seed, table_slots, parent, max_probe,
-                               host_staging)
+                               host_staging, deterministic)
         need = workspace_bytes(self.cfg)
         if need == 0:
             raise StandError("invalid configuration")

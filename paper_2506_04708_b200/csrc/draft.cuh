@@ -33,6 +33,7 @@ struct DraftParams {
   int* cand_id;            // [B, N, K]
   float* cand_phi;         // [B, N, K]
   unsigned long long* stats;
+  int deterministic;       // != 0: the children are the most probable candidates, no noise
 };
 
 // Rank of this lane's candidate by g = log(phi) - log(-log U) in double precision (larger first, equal
@@ -134,9 +135,10 @@ __global__ void __launch_bounds__(K4_THREADS) draft_kernel(const DraftParams p) 
       // Perturbed scores in single precision first; they decide the order whenever every pair of
       // candidates is further apart than single precision can blur (1e-3 against errors of a few 1e-6).
       // Otherwise the scores are formed again in double precision.
-      const uint32_t u24 = valid ? philox_u24(p.seed, b, p.step, u, SLOT_GUMBEL | (uint32_t)id) : 0u;
+      const uint32_t u24 = (valid && !p.deterministic) ? philox_u24(p.seed, b, p.step, u, SLOT_GUMBEL | (uint32_t)id) : 0u;
       float gf = 0.0f;
-      if (valid) {
+      if (valid && p.deterministic) gf = phi;  // deterministic drafting (Sec. 3.2): rank by the stored probability itself
+      else if (valid) {
         // L = -log U with U = (u24 + 1/2) / 2^24.  Below one half U is exact in fp32 and the hardware
         // logarithm serves; above, L = 2 atanh(v / (2 - v)) with the exact complement v = 1 - U <= 1/2.
         const float lo = -__logf(((float)u24 + 0.5f) * (1.0f / 16777216.0f));
@@ -162,7 +164,7 @@ __global__ void __launch_bounds__(K4_THREADS) draft_kernel(const DraftParams p) 
         }
       }
       __syncwarp();
-      if (__any_sync(FULL, valid && close)) rank = gumbel_rank_double(valid, id, phi, u24);
+      if (!p.deterministic && __any_sync(FULL, valid && close)) rank = gumbel_rank_double(valid, id, phi, u24);
       if (valid && rank < m) s_tok[s_fc[u] + rank] = id;
       const unsigned vmask = __ballot_sync(FULL, valid);
       if (valid) {

@@ -38,7 +38,7 @@ bool derive(const stand_config* c, Derived* d) {
   if (c->B < 1 || c->N < 1 || c->N > STAND_MAX_NODES || c->V < 2 || c->V > STAND_MAX_VOCAB) return false;
   if (c->topk < 1 || c->topk > STAND_MAX_TOPK || c->order_max < 1 || c->order_max > STAND_MAX_ORDER) return false;
   if (c->dtype != STAND_DTYPE_F32 && c->dtype != STAND_DTYPE_BF16) return false;
-  if (!(c->temperature > 0.0f) || c->max_probe < 0 || c->reserved != 0) return false;
+  if (!(c->temperature > 0.0f) || c->max_probe < 0 || (c->deterministic != 0 && c->deterministic != 1)) return false;
   if (c->table_slots < 2 || (c->table_slots & (c->table_slots - 1)) != 0 || c->table_slots > (1ull << 32) - 2) return false;
   if (!c->parent || c->parent[0] != -1) return false;
   if ((long long)c->B * c->N > (1ll << 31) / 4) return false;
@@ -252,6 +252,7 @@ int run_verify(stand_ctx* x, const void* logits, int32_t* emitted, int32_t* n_em
   v.rec_ctx = x->at<int>(x->L.rec_ctx); v.rec_ids = x->at<int>(x->L.rec_ids); v.rec_p = x->at<float>(x->L.rec_p);
   v.stats = x->at<unsigned long long>(x->L.stats);
   v.node_accepts = x->at<unsigned long long>(x->L.accepts);
+  v.deterministic = c.deterministic;
   v.fuse_locate = fuse_locate ? 1 : 0;
   v.upd = step_update_params(x);
   // inside a fused step (and with no timing events between the launches) the kernels chain programmatically
@@ -299,6 +300,7 @@ int run_draft(stand_ctx* x, int32_t* tree_user, bool chained, cudaStream_t st) {
   d.level_start = x->topo_level_start(); d.tail = x->at<int>(x->L.tail); d.tree = x->at<int>(x->L.tree);
   d.tree_user = tree_user; d.cand_n = x->at<int>(x->L.cand_n); d.cand_id = x->at<int>(x->L.cand_id);
   d.cand_phi = x->at<float>(x->L.cand_phi); d.stats = x->at<unsigned long long>(x->L.stats);
+  d.deterministic = c.deterministic;
   int rc;
   if (chained && !x->ev_stage[3]) rc = launch_dependent(draft_kernel, (unsigned)c.B, K4_THREADS, st, d);
   else { draft_kernel<<<c.B, K4_THREADS, 0, st>>>(d); rc = launch_ok(); }

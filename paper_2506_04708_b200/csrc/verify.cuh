@@ -52,6 +52,7 @@ struct VerifyParams {
   float* rec_p;            // [B, D+1, K]
   unsigned long long* stats;
   unsigned long long* node_accepts;  // [N] how often each node lay on an accepted path
+  int deterministic;       // != 0: deterministic drafting (every drafted token is a one-hot draft)
   int fuse_locate;         // != 0: also run stage 1 of the N-gram update for this sequence's records
   UpdateParams upd;        // used when fuse_locate is set
 };
@@ -358,6 +359,13 @@ __global__ void __launch_bounds__(K2_THREADS, 2) verify_kernel(const VerifyParam
         const double U = __shfl_sync(FULL, Uj, j & 15);
         const double qx = __shfl_sync(FULL, qh, ix < 0 ? 0 : ix);
         const double px = __shfl_sync(FULL, ph, ix < 0 ? 0 : ix);
+        if (p.deterministic) {
+          // one-hot draft: accept iff U < p~(x); on rejection x loses its mass and the rest is renormalised
+          if (ix < 0 || U * zr < px) { accepted = j; break; }
+          zr -= px;
+          if (li == ix) ph = 0.0;
+          continue;
+        }
         if (ix < 0 || U * qx * zr < px * qn) { accepted = j; break; }
         const double a = ph * qn, c2 = qh * zr;
         const double ov = half_sum_d(fmin(a, c2));

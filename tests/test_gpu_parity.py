@@ -132,6 +132,46 @@ def test_tiny_shapes(V, N, D, kb, dtype):
     _run(w, 60, "p80", check_every=20)
 
 
+# ------------------------------------------------------------ deterministic drafting (Sec. 3.2)
+@pytest.mark.parametrize("dtype", [inputs.DTYPE_F32, inputs.DTYPE_BF16])
+def test_deterministic_drafting_small(dtype):
+    w = inputs.Workload("det", 4, 16, 4, 3, 3000, dtype, 0.8, 3, 8, 120, 1 << 14, 2.0, 0.7, 16, 1.1)
+    acc, _, st = _run(w, 120, "p80", check_every=40, deterministic=True)
+    assert acc > 1.1 and sum(st["lookup_hits"]) > 0
+
+
+def test_deterministic_drafting_cfg3_window():
+    _run(inputs.WORKLOADS["cfg3"], 8, "p80", table_slots=1 << 16, check_every=4, deterministic=True)
+
+
+def test_deterministic_and_stochastic_drafting_differ_only_in_the_draft():
+    """Same seeds, same logits: before any tree exists both modes emit the same first token; afterwards the
+    deterministic tree holds the most probable candidates of each lookup."""
+    torch = _torch()
+    from paper_2506_04708_b200.binding import Stand
+    w = inputs.scaled(inputs.WORKLOADS["cfg1"], B=2)
+    parent = inputs.topology(w.N, w.D, w.kb)
+    depth = inputs.node_depths(parent)
+    streams = inputs.token_streams(w, 5, 300)
+    a = Stand(w.B, w.N, w.V, w.topk, w.order_max, w.dtype, w.T, 5, 1 << 12, parent)
+    b = Stand(w.B, w.N, w.V, w.topk, w.order_max, w.dtype, w.T, 5, 1 << 12, parent, deterministic=True)
+    tail = torch.from_numpy(streams[:, 5:8].copy())
+    lens = np.full(w.B, 8, np.int64)
+    for g in (a, b):
+        g.reset_sequences(tail, torch.from_numpy(lens))
+    dl = harness.to_device_logits(inputs.logits_numpy(w, streams, lens, depth, 0, 5, "p80"))
+    ea, _, ta = (t.cpu().numpy().copy() for t in a.step(dl))
+    eb, _, tb = (t.cpu().numpy().copy() for t in b.step(dl))
+    assert np.array_equal(ea, eb)              # no tree yet: one token from the root row, same uniform
+    st = b.state_dump()
+    for s in range(w.B):                        # the first child of the root is the most probable candidate
+        n = st["cand_n"][s, 0]
+        if n:
+            best = st["cand_id"][s, 0, np.lexsort((st["cand_id"][s, 0, :n], -st["cand_phi"][s, 0, :n]))[0]]
+            assert tb[s, 1] == best
+    a.close(); b.close()
+
+
 # ------------------------------------------------ acceptance counters and tree optimisation (Sec. 4.2)
 def test_node_acceptance_counters_and_tree_optimisation():
     """Data-driven tree optimisation on a synthetic workload: start from (a 128-node prefix of) Algorithm 1's
