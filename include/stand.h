@@ -153,8 +153,9 @@ int stand_step_host(stand_ctx* ctx, const void* host_logits, int32_t* host_emitt
  * x/T (dev_lse [rows] float), and the top-k entries by (value descending, id
  * ascending): dev_ids [rows, topk] int32, dev_values [rows, topk] float (input
  * values), dev_probs [rows, topk] float (softmax probabilities).  dev_scratch must
- * hold stand_row_stats_scratch_bytes bytes, 256-byte aligned.  Inputs are finite or
- * -inf.  If a bounded wait inside the kernel runs out (never seen; it guards against a
+ * hold stand_row_stats_scratch_bytes bytes, 256-byte aligned.  Inputs are -inf or
+ * finite with |x| * log2(e) / T < 2^24 (beyond that the fp32 exponent offsets lose their
+ * integer precision); the same holds for every entry point that takes logits.  If a bounded wait inside the kernel runs out (never seen; it guards against a
  * hang), every dev_lse entry is NaN and every id -1. */
 size_t stand_row_stats_scratch_bytes(int64_t rows, int32_t V, int32_t dtype, int32_t topk);
 int stand_row_stats(const void* dev_logits, int64_t rows, int32_t V, int32_t dtype, float temperature, int32_t topk,

@@ -57,6 +57,66 @@ def test_row_stats_unaligned_rows_and_many_rows():
             assert np.allclose(probs[r], oprobs, rtol=1e-5 if raw.dtype == np.float32 else 4e-3)
 
 
+def test_row_stats_degenerate_rows():
+    """Rows that defeat the chunk-maximum bound: constant rows (every entry reaches the bound, so the candidate
+    buffers overflow and the streaming selection takes over), rows with -inf, and one-entry maxima."""
+    from paper_2506_04708_b200 import binding
+    V, k = 5000, 10
+    x = np.zeros((6, V), np.float32)
+    x[0, :] = 1.5                                  # constant: top-k = the first k ids
+    x[1, :] = -np.inf; x[1, 4321] = 0.25           # a single finite entry
+    x[2, :] = np.arange(V) % 7                     # long runs of equal maxima in every chunk
+    x[3, :] = -np.inf; x[3, :3] = [1.0, 2.0, 3.0]  # fewer finite entries than k
+    x[4, :] = -1e6; x[4, V - 1] = 1e6              # extreme spread (the documented range is |x| log2(e) / T < 2^24)
+    x[5, :] = -0.0; x[5, ::2] = 0.0                # +0 and -0 are one value: ties by id
+    for raw in (x, inputs.f32_to_bf16_bits(x)):
+        tol = 1e-5 if raw.dtype == np.float32 else 4e-3
+        lse, ids, vals, probs = (t.cpu().numpy() for t in binding.row_stats(harness.to_device_logits(raw), 1.0, k))
+        for r in range(x.shape[0]):
+            olse, oids, ovals, oprobs, _ = so.row_stats(raw[r], 1.0, k)
+            assert np.array_equal(ids[r], oids), (r, ids[r], oids)
+            assert abs(lse[r] - olse) <= 1e-5 * max(1.0, abs(olse)), (r, lse[r], olse)
+            assert np.allclose(probs[r], oprobs, rtol=tol, atol=1e-30), r
+
+
+def test_maximum_sizes():
+    """The largest vocabulary (2^20: 1024 chunks, the general bound search), the largest tree (128 nodes), top-12,
+    order 4: a few whole steps against the oracle."""
+    parent = inputs.topology(128, 8, 4)
+    w = inputs.Workload("max", 2, 128, 8, 4, 1 << 20, inputs.DTYPE_BF16, 0.7, 4, 12, 3, 1 << 14, 2.5, 0.6, 32, 1.05)
+    loop = harness.ClosedLoop(w, seed=1, peak_mode="add8", parent=parent, device_logits=True)
+    try:
+        for _ in range(w.steps):
+            loop.step()
+        assert loop.hard == [] and loop.check_state_and_table() == []
+        assert loop.gpu.stats()["wait_timeouts"] == 0
+    finally:
+        loop.close()
+
+
+def test_constant_logits_through_the_whole_step():
+    """Every row constant: the uniform target distribution, all top-k ties broken by id, through verify, update, draft."""
+    torch = _torch()
+    from paper_2506_04708_b200.binding import Stand
+    w = inputs.scaled(inputs.WORKLOADS["cfg1"], B=2, V=3000)
+    parent = inputs.topology(w.N, w.D, w.kb)
+    gpu = Stand(w.B, w.N, w.V, w.topk, w.order_max, w.dtype, w.T, 3, 1 << 12, parent)
+    orc = so.Oracle(w.B, w.N, w.V, w.topk, w.order_max, w.dtype, w.T, 3, parent)
+    tail = np.array([[1, 2, 3], [4, 5, 6]], np.int32)
+    lens = np.full(w.B, 8, np.int64)
+    gpu.reset_sequences(torch.from_numpy(tail), torch.from_numpy(lens))
+    orc.reset_sequences(tail, lens)
+    logits = np.full((w.B, w.N, w.V), 0.5, np.float32)
+    for s in range(4):
+        em, ne, tr = (t.cpu().numpy() for t in gpu.step(harness.to_device_logits(logits)))
+        em_o, ne_o, tr_o = orc.step(logits)
+        _, margins = orc.take_margins()
+        if margins.size == 0 or margins.min() >= harness.MARGIN_TOL:
+            assert np.array_equal(em, em_o) and np.array_equal(ne, ne_o) and np.array_equal(tr, tr_o), s
+    assert harness.compare_tables(gpu.table_dict(), orc.table(), 1e-5) == []
+    gpu.close(); orc.close()
+
+
 # ------------------------------------------------------------- whole step, closed loop
 def _run(w, steps, peak_mode, seed=0, check_every=0, **kw):
     w = inputs.scaled(w, steps=steps)
