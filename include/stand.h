@@ -40,7 +40,7 @@ extern "C" {
 
 #define STAND_MAX_TOPK 12   /* entries kept per context (one 128-byte table slot) */
 #define STAND_MAX_ORDER 4   /* N-gram orders 1..4 (Sec. 4.1) */
-#define STAND_MAX_NODES 128 /* tree nodes per sequence */
+#define STAND_MAX_NODES 640 /* tree nodes per sequence (Algorithm 1's initial tree has 625) */
 #define STAND_MAX_DEPTH 32
 #define STAND_MAX_VOCAB (1 << 20)
 

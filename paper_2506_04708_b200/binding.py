@@ -12,7 +12,7 @@ import numpy as np
 _PKG = os.path.dirname(os.path.abspath(__file__))
 LIB_PATH = os.path.join(_PKG, "libstand.so")
 
-STAND_MAX_TOPK, STAND_MAX_ORDER, STAND_MAX_NODES = 12, 4, 128
+STAND_MAX_TOPK, STAND_MAX_ORDER, STAND_MAX_NODES = 12, 4, 640
 DTYPE_F32, DTYPE_BF16 = 0, 1
 
 EXPORTS = [

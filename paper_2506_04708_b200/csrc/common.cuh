@@ -10,7 +10,7 @@ constexpr unsigned FULL = 0xFFFFFFFFu;
 constexpr int CHUNK = 1024;  // vocabulary entries per chunk: one (sum, offset) pair each
 constexpr int KMAX = 12;     // STAND_MAX_TOPK
 constexpr int ORDER_MAX = 4; // STAND_MAX_ORDER
-constexpr int NODES_MAX = 128;
+constexpr int NODES_MAX = 640;  // STAND_MAX_NODES
 constexpr int DEPTH_MAX = 32;
 constexpr int VOCAB_MAX = 1 << 20;  // STAND_MAX_VOCAB
 

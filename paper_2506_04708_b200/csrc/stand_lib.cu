@@ -155,6 +155,10 @@ int prepare_device(int* sm_count) {
     if (cudaFuncSetAttribute(row_pass_kernel<1, K1Shape<1>::CW, K1_CTAS>, cudaFuncAttributeMaxDynamicSharedMemorySize,
                              k1_smem_bytes<1>()) != cudaSuccess)
       return STAND_E_CUDA;
+    // large trees keep their per-node state in more shared memory than the default limit
+    if (cudaFuncSetAttribute(verify_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)verify_smem_bytes(NODES_MAX)) !=
+        cudaSuccess)
+      return STAND_E_CUDA;
     g_sm_count[dev].store(sms, std::memory_order_relaxed);
     g_k1_ready[dev].store(1, std::memory_order_release);
   }
@@ -257,8 +261,9 @@ int run_verify(stand_ctx* x, const void* logits, int32_t* emitted, int32_t* n_em
   v.upd = step_update_params(x);
   // inside a fused step (and with no timing events between the launches) the kernels chain programmatically
   const bool chain = fuse_locate && !x->ev_after && !x->ev_stage[1];
-  if (chain) rc = launch_dependent(verify_kernel, (unsigned)c.B, K2_THREADS, st, v);
-  else { verify_kernel<<<c.B, K2_THREADS, 0, st>>>(v); rc = launch_ok(); }
+  const size_t vsm = verify_smem_bytes(c.N);
+  if (chain) rc = launch_dependent(verify_kernel, (unsigned)c.B, K2_THREADS, st, v, vsm);
+  else { verify_kernel<<<c.B, K2_THREADS, vsm, st>>>(v); rc = launch_ok(); }
   if (rc) return rc;
   if (x->ev_stage[2]) cudaEventRecord(x->ev_stage[2], st);
   x->launches += 1;
@@ -337,6 +342,11 @@ int stand_init(const stand_config* cfg, void* dev_workspace, size_t bytes, stand
   Layout L;
   layout_of(cfg, &d, &L);
   if (!dev_workspace || ((uintptr_t)dev_workspace & 255) != 0 || bytes < L.total) return STAND_E_WORKSPACE;
+  {
+    int sms = 0;
+    const int prc = prepare_device(&sms);  // kernel attributes of this device, once
+    if (prc) return prc;
+  }
   stand_ctx* x = new (std::nothrow) stand_ctx;
   if (!x) return STAND_E_ARG;
   x->cfg = *cfg;

@@ -85,6 +85,11 @@ constexpr int TOPK_ROWS = 4;       // path rows whose top-k is selected together
 constexpr int TOPK_ITEMS = 1024;   // (row, chunk) work items per group of rows
 constexpr int ROW_LANES = 8;       // lanes that share one row in the normaliser phase
 
+// Dynamic shared memory of the verification kernel for a tree of N nodes.
+inline size_t verify_smem_bytes(int N) {
+  return (size_t)N * (KMAX * (sizeof(double) + sizeof(float) + sizeof(int)) + sizeof(double) + sizeof(float) + 4 * sizeof(int));
+}
+
 // Pushes the entries of chunk `ch` of a row that reach `floor` into buf (capacity cap; *cnt keeps
 // counting past it, which the caller reads as overflow).  Called by all lanes of a warp.
 __device__ __forceinline__ void push_chunk_candidates(const void* logits, int dtype, long long row, int V, int ch,
@@ -232,12 +237,18 @@ __device__ __forceinline__ double half_sum_d(double v) {
 }
 
 __global__ void __launch_bounds__(K2_THREADS, 2) verify_kernel(const VerifyParams p) {
-  __shared__ float s_off[NODES_MAX];
-  __shared__ double s_invZ[NODES_MAX];
-  __shared__ double s_p[NODES_MAX][KMAX];  // target probability of candidate i of node u
-  __shared__ int s_tree[NODES_MAX], s_cn[NODES_MAX], s_fc[NODES_MAX], s_nch[NODES_MAX];
-  __shared__ int s_cid[NODES_MAX][KMAX];
-  __shared__ float s_cphi[NODES_MAX][KMAX];
+  // per-node state, sized by the tree (verify_smem_bytes): target probabilities of the candidates, normaliser
+  // reciprocals and offsets, the candidate lists, tree tokens and topology
+  extern __shared__ __align__(16) unsigned char s_dyn[];
+  double* s_p = reinterpret_cast<double*>(s_dyn);                 // [N][KMAX]
+  double* s_invZ = s_p + (size_t)p.N * KMAX;                      // [N]
+  float* s_off = reinterpret_cast<float*>(s_invZ + p.N);          // [N]
+  float* s_cphi = s_off + p.N;                                    // [N][KMAX]
+  int* s_cid = reinterpret_cast<int*>(s_cphi + (size_t)p.N * KMAX);  // [N][KMAX]
+  int* s_tree = s_cid + (size_t)p.N * KMAX;                       // [N]
+  int* s_cn = s_tree + p.N;
+  int* s_fc = s_cn + p.N;
+  int* s_nch = s_fc + p.N;
   __shared__ int s_tail[ORDER_MAX];
   __shared__ double s_scan[K2_THREADS / 32];
   __shared__ int s_path[DEPTH_MAX + 1];
@@ -271,22 +282,23 @@ __global__ void __launch_bounds__(K2_THREADS, 2) verify_kernel(const VerifyParam
   }
   for (int i = tid; i < N * K; i += K2_THREADS) {
     const int u = i / K, t = i - u * K;
-    s_cid[u][t] = p.cand_id[(long long)b * N * K + i];
-    s_cphi[u][t] = p.cand_phi[(long long)b * N * K + i];
+    s_cid[(u) * KMAX + (t)] = p.cand_id[(long long)b * N * K + i];
+    s_cphi[(u) * KMAX + (t)] = p.cand_phi[(long long)b * N * K + i];
   }
   if (tid < p.n_max) s_tail[tid] = p.tail[b * p.n_max + tid];
   __syncthreads();
 
   // ---- phase 1: the candidate logits are requested first (one round of gathers), the normalisers
   // (8 lanes per row) are formed while they travel ----
-  constexpr int GATHERS = NODES_MAX * KMAX / K2_THREADS;
+  // (trees of up to 128 nodes are covered by these six gathers per thread; larger ones gather again below)
+  constexpr int GATHERS = 128 * KMAX / K2_THREADS;
   float gx[GATHERS];
 #pragma unroll
   for (int k = 0; k < GATHERS; ++k) {
     const int i = tid + k * K2_THREADS;
     const int u = i / KMAX, t = i - u * KMAX;
     gx[k] = 0.0f;
-    if (u < N && t < s_cn[u]) gx[k] = load_logit(p.logits, p.dtype, ((long long)b * N + u) * (long long)p.V + s_cid[u][t]);
+    if (u < N && t < s_cn[u]) gx[k] = load_logit(p.logits, p.dtype, ((long long)b * N + u) * (long long)p.V + s_cid[(u) * KMAX + (t)]);
   }
   pdl_wait();  // the chunk pairs come from the row pass
   {
@@ -318,7 +330,14 @@ __global__ void __launch_bounds__(K2_THREADS, 2) verify_kernel(const VerifyParam
   for (int k = 0; k < GATHERS; ++k) {
     const int i = tid + k * K2_THREADS;
     const int u = i / KMAX, t = i - u * KMAX;
-    if (u < N && t < s_cn[u]) s_p[u][t] = exp2_d((double)gx[k] * cd - (double)s_off[u]) * s_invZ[u];
+    if (u < N && t < s_cn[u]) s_p[(u) * KMAX + (t)] = exp2_d((double)gx[k] * cd - (double)s_off[u]) * s_invZ[u];
+  }
+  for (int i = tid + GATHERS * K2_THREADS; i < N * KMAX; i += K2_THREADS) {  // the rest of a large tree
+    const int u = i / KMAX, t = i - u * KMAX;
+    if (t < s_cn[u]) {
+      const float x = load_logit(p.logits, p.dtype, ((long long)b * N + u) * (long long)p.V + s_cid[(u) * KMAX + (t)]);
+      s_p[(u) * KMAX + (t)] = exp2_d((double)x * cd - (double)s_off[u]) * s_invZ[u];
+    }
   }
   __syncthreads();
 
@@ -345,9 +364,9 @@ __global__ void __launch_bounds__(K2_THREADS, 2) verify_kernel(const VerifyParam
       scale = 1.0;
       if (drafted <= 0) break;  // nothing drafted below u: sample from its target
       const int nc = s_cn[u];
-      const int cid = li < nc ? s_cid[u][li] : -1;
-      double ph = li < nc ? s_p[u][li] : 0.0;
-      double qh = li < nc ? (double)s_cphi[u][li] : 0.0;
+      const int cid = li < nc ? s_cid[(u) * KMAX + (li)] : -1;
+      double ph = li < nc ? s_p[(u) * KMAX + (li)] : 0.0;
+      double qh = li < nc ? (double)s_cphi[(u) * KMAX + (li)] : 0.0;
       double qn = half_sum_d(qh), zr = 1.0, pq = 1.0;
       // the uniforms of all children at once
       const double Uj = li < drafted ? (double)philox_u24(p.seed, b, p.step, u, (uint32_t)li) * (1.0 / 16777216.0) : 0.0;
@@ -385,7 +404,7 @@ __global__ void __launch_bounds__(K2_THREADS, 2) verify_kernel(const VerifyParam
       const double inv = 1.0 / zr;
       scale = pq * inv;
       nsup = nc;
-      if (lane < nc) { s_sup_id[lane] = cid; s_sup_pt[lane] = ph * inv; s_sup_p[lane] = s_p[u][lane]; }
+      if (lane < nc) { s_sup_id[lane] = cid; s_sup_pt[lane] = ph * inv; s_sup_p[lane] = s_p[(u) * KMAX + (lane)]; }
       break;
     }
     if (lane == 0) {

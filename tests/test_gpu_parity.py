@@ -271,6 +271,36 @@ def test_node_acceptance_counters_and_tree_optimisation():
         loop2.close()
 
 
+def test_full_initial_tree_to_eighty_nodes():
+    """The paper's procedure at its own sizes (Sec. 4.2, App. A.1): all 625 nodes of Algorithm 1's tree, acceptance
+    counts over a run, the 80 most accepted nodes kept."""
+    from paper_2506_04708_b200 import binding
+    parent, depth, _, total = binding.initial_tree()
+    assert total == 625 and len(parent) == 625
+    w = inputs.Workload("init625", 3, 625, int(depth.max()), 8, 2000, inputs.DTYPE_BF16, 0.6, 4, 10, 25, 1 << 14, 2.0, 0.7,
+                        24, 1.05)
+    loop = harness.ClosedLoop(w, seed=4, peak_mode="p80", parent=parent)
+    try:
+        for _ in range(w.steps):
+            loop.step()
+        assert loop.hard == [] and loop.check_state_and_table() == []
+        got = loop.gpu.node_accepts()
+        assert got[0] == w.B * w.steps
+        small, old = binding.prune_tree(parent, got, 80)
+    finally:
+        loop.close()
+    assert len(small) == 80 and small[0] == -1
+    w2 = inputs.Workload("opt80", 3, 80, int(inputs.node_depths(small).max()), 8, 2000, inputs.DTYPE_BF16, 0.6, 4, 10, 20,
+                         1 << 14, 2.0, 0.7, 24, 1.05)
+    loop2 = harness.ClosedLoop(w2, seed=4, peak_mode="p80", parent=small)
+    try:
+        for _ in range(w2.steps):
+            loop2.step()
+        assert loop2.hard == [] and loop2.check_state_and_table() == []
+    finally:
+        loop2.close()
+
+
 # ------------------------------------------------------------------- stages on their own
 def test_stage_calls_equal_the_fused_step():
     torch = _torch()
