@@ -192,6 +192,12 @@ def test_tiny_shapes(V, N, D, kb, dtype):
     _run(w, 60, "p80", check_every=20)
 
 
+def test_more_sequences_than_resident_blocks():
+    """Many more sequences than the GPU holds thread blocks at once: several waves of every per-sequence kernel."""
+    w = inputs.Workload("wide", 700, 4, 2, 2, 200, inputs.DTYPE_F32, 0.9, 2, 6, 12, 1 << 14, 2.0, 0.7, 12, 1.1)
+    _run(w, 12, "p80", check_every=6)
+
+
 # ------------------------------------------------------------ deterministic drafting (Sec. 3.2)
 @pytest.mark.parametrize("dtype", [inputs.DTYPE_F32, inputs.DTYPE_BF16])
 def test_deterministic_drafting_small(dtype):
