@@ -338,6 +338,46 @@ def test_stage_calls_equal_the_fused_step():
     a.close(); b.close()
 
 
+def test_table_persists_across_trajectories_and_resume_from_a_checkpoint():
+    """Sec. 5.1: the N-gram module is kept across trajectories (stand_reset_sequences restarts the sequences only).
+    And a run resumed in a fresh context from dumped table + state continues exactly like the original."""
+    torch = _torch()
+    from paper_2506_04708_b200.binding import Stand
+    w = inputs.scaled(inputs.WORKLOADS["cfg1"], B=3, V=4000, steps=40)
+    loop = harness.ClosedLoop(w, seed=9, peak_mode="p80", table_slots=1 << 14)
+    try:
+        for _ in range(20):
+            loop.step()
+        n_ctx = len(loop.orc.table())
+        # a new trajectory: same prompts, sequences restart, the table stays
+        tail = np.full((w.B, w.order_max), -1, np.int32)
+        tail[:, :] = loop.streams[:, 8 - w.order_max:8]
+        lens = np.full(w.B, 8, np.int64)
+        loop.gpu.reset_sequences(torch.from_numpy(tail), torch.from_numpy(lens))
+        loop.orc.reset_sequences(tail, lens)
+        loop.lens = lens
+        assert len(loop.gpu.table_dict()) == n_ctx
+        for _ in range(10):
+            loop.step()
+        assert loop.hard == [] and loop.check_state_and_table() == []
+        assert len(loop.orc.table()) >= n_ctx and sum(loop.gpu.stats()["lookup_hits"]) > 0
+        # checkpoint, resume elsewhere, and run both on the same logits
+        other = Stand(w.B, w.N, w.V, w.topk, w.order_max, w.dtype, w.T, 9, 1 << 15, loop.parent)
+        other.table_load(*loop.gpu.table_dump())
+        other.state_load(loop.gpu.state_dump())
+        for s in range(5):
+            logits = inputs.logits_numpy(w, loop.streams, loop.lens, loop.depth, 100 + s, 9, "p80")
+            dl = harness.to_device_logits(logits)
+            a = [t.cpu().numpy().copy() for t in loop.gpu.step(dl)]
+            b = [t.cpu().numpy().copy() for t in other.step(dl)]
+            assert all(np.array_equal(x, y) for x, y in zip(a, b)), s
+            loop.lens = loop.gpu.state_dump()["len"]
+        assert other.table_dict() == loop.gpu.table_dict()
+        other.close()
+    finally:
+        loop.close()
+
+
 def test_bulk_update_and_table_roundtrip():
     torch = _torch()
     from paper_2506_04708_b200.binding import Stand
