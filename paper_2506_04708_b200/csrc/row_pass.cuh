@@ -9,8 +9,8 @@
 // (Sec. 4.1) so tightly that it can be finished afterwards from about k chunks, for
 // the few rows that need it (row_topk_warp below).
 //
-// The kernel is bound by HBM bandwidth: persistent CTAs (two per SM) walk a
-// contiguous range of tiles (16 chunks for bf16, 8 for fp32); one elected lane
+// The kernel is bound by HBM bandwidth: persistent CTAs (one per SM) walk a
+// contiguous range of tiles (31 chunks for bf16, 16 for fp32: about 64 KB); one elected lane
 // streams tiles into a ring of shared-memory stages with bulk asynchronous copies
 // (TMA) that complete on mbarriers, marked evict-first in L2; each consumer warp
 // takes one chunk of every tile.  The inner loop has no branches: packed bf16 max, packed fp32 FMA/ADD,
@@ -20,13 +20,17 @@
 
 namespace stand {
 
-constexpr int K1_SMEM_DATA = 96 * 1024;  // ring bytes per CTA at two CTAs per SM
-constexpr int K1_CTAS = 2;               // persistent CTAs per SM
-// consumer warps per CTA = chunks per tile: bf16 needs 32 warps per SM to keep the exp unit fed (16 per CTA:
-// 6.6 TB/s against 6.2 TB/s with 8); fp32 moves twice the bytes per exp and is fed by 8.
-template <int DT> struct K1Shape { static constexpr int CW = DT == 1 ? 16 : 8; };
+constexpr int K1_SMEM_DATA = 96 * 1024;  // ring bytes per SM = 2 * K1_SMEM_DATA, shared by the CTAs of an SM
+constexpr int K1_CTAS = 1;               // persistent CTAs per SM
+// Consumer warps per CTA = chunks per tile.  Measured on 1.9 - 2.1 GB: large bulk copies win (bf16: one CTA of 31
+// consumer warps, 62 KB tiles, 6.81 TB/s; two CTAs of 16 warps, 32 KB tiles, 6.60; of 8 warps, 16 KB tiles, 6.2;
+// fp32: 16 warps and 64 KB tiles 6.73 against 6.55 with 8 and 32 KB), as long as about 32 warps per SM keep the
+// exp unit fed for bf16.  31 consumer warps + the producer warp fill a 1024-thread block.
+template <int DT> struct K1Shape { static constexpr int CW = DT == 1 ? 31 : 16; };
 template <int DT> constexpr int k1_stage_bytes() { return K1Shape<DT>::CW * CHUNK * (DT == 1 ? 2 : 4); }
-template <int DT> constexpr int k1_smem_bytes() { return (K1_SMEM_DATA / k1_stage_bytes<DT>()) * k1_stage_bytes<DT>(); }
+template <int DT> constexpr int k1_smem_bytes() {
+  return (2 * K1_SMEM_DATA / K1_CTAS / k1_stage_bytes<DT>()) * k1_stage_bytes<DT>();
+}
 constexpr unsigned SPIN_LIMIT = 1u << 22;                  // bounded waits: about a second, then the kernel gives up
 
 constexpr int COMPACT_AT = 64;              // candidate count that triggers a compaction
