@@ -302,7 +302,8 @@ struct SlotImage {
 // Lanes exchange their pairs through shared memory rather than shuffles: a lane reads the other pairs
 // with independent loads, which a single warp overlaps, where a chain of shuffles costs its full
 // latency each (measured: 3,000 cycles per merge with shuffles and match_any, a few hundred this way).
-__device__ __forceinline__ void merge_warp(SlotImage* img, const int* f_ids, const float* f_p, int K, int lane) {
+// The fresh row arrives in registers: lane 16 + t carries entry t (fid < 0: none).
+__device__ __forceinline__ void merge_warp(SlotImage* img, int fid, float fp, int K, int lane) {
   const double c = (double)img->count;
   const double w_old = c / (c + 1.0), w_new = 1.0 / (c + 1.0);
   const int n_items = (int)img->n_items;
@@ -311,8 +312,7 @@ __device__ __forceinline__ void merge_warp(SlotImage* img, const int* f_ids, con
   if (lane < KMAX) {
     if (lane < n_items) { id = img->ids[lane]; val = __dmul_rn((double)img->probs[lane], w_old); }
   } else if (lane >= 16 && lane < 16 + K) {
-    const int fid = f_ids[lane - 16];
-    if (fid >= 0) { id = fid; val = __dmul_rn((double)f_p[lane - 16], w_new); }
+    if (fid >= 0) { id = fid; val = __dmul_rn((double)fp, w_new); }
   }
   img->m_id[lane] = id;
   img->m_val[lane] = val;
@@ -351,6 +351,16 @@ __device__ __forceinline__ void merge_warp(SlotImage* img, const int* f_ids, con
 // applies all records of that slot in row order (the canonical order of same-step
 // updates) and closes the slot's update fields.
 constexpr int APPLY_WARPS = 8;
+// Entry t of compressed row i for lane 16 + t (other lanes: none).
+__device__ __forceinline__ void load_fresh(const UpdateParams& p, long long i, int lane, int& fid, float& fp) {
+  fid = -1;
+  fp = 0.0f;
+  if (lane >= 16 && lane < 16 + p.K) {
+    fid = p.rec_ids[i * p.K + (lane - 16)];
+    fp = p.rec_p[i * p.K + (lane - 16)];
+  }
+}
+
 __global__ void __launch_bounds__(APPLY_WARPS * 32) update_apply_kernel(const UpdateParams p) {
   __shared__ SlotImage s_img[APPLY_WARPS];
   const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
@@ -362,49 +372,70 @@ __global__ void __launch_bounds__(APPLY_WARPS * 32) update_apply_kernel(const Up
   const int n = (int)(g / p.n_rows) + 1;
   const long long row = g - (long long)(n - 1) * p.n_rows;
   const uint32_t* seg = p.rec_slot + (long long)(n - 1) * p.n_rows;
+  // one round trip: the record's slot, its compressed row, and the first window of later records
   const uint32_t slot = seg[row];
+  int fid;
+  float fp;
+  load_fresh(p, row, lane, fid, fp);
+  constexpr int WIN = 4;
+  long long i0 = (row + 1) & ~31ll;
+  uint32_t got[WIN];
+#pragma unroll
+  for (int w = 0; w < WIN; ++w) {
+    const long long i = i0 + 32 * w + lane;
+    got[w] = (i > row && i < p.n_rows) ? seg[i] : NO_SLOT;
+  }
   if (slot == NO_SLOT) return;
-  Slot* s = &p.table[slot];
-  if (s->lead != (uint32_t)row) return;  // another record leads this slot
-  const uint32_t pending = s->pend;
+  // second round trip: the whole 128-byte slot, one word per lane (key 0-3, count, n_items, lead, pend, ids, probs)
+  uint32_t* line = reinterpret_cast<uint32_t*>(&p.table[slot]);
+  const uint32_t word = line[lane];
+  if (__shfl_sync(FULL, word, 6) != (uint32_t)row) return;  // another record leads this slot
+  const uint32_t pending = __shfl_sync(FULL, word, 7);
   SlotImage* img = &s_img[warp];
-  if (lane == 0) { img->count = s->count; img->n_items = s->n_items; }
-  if (lane < KMAX) { img->ids[lane] = s->ids[lane]; img->probs[lane] = s->probs[lane]; }
+  if (lane == 4) img->count = word;
+  if (lane == 5) img->n_items = word;
+  if (lane >= 8 && lane < 8 + KMAX) img->ids[lane - 8] = (int)word;
+  if (lane >= 8 + KMAX) img->probs[lane - 8 - KMAX] = __uint_as_float(word);
   __syncwarp();
   const bool fresh_slot = img->count == 0;
-  merge_warp(img, p.rec_ids + row * p.K, p.rec_p + row * p.K, p.K, lane);
+  merge_warp(img, fid, fp, p.K, lane);
   uint32_t applied = 1;
-  // the other records of this slot, in row order; four 32-wide windows of rec_slot are in flight at once
-  constexpr int WIN = 4;
-  for (long long i0 = (row + 1) & ~31ll; applied < pending && i0 < p.n_rows; i0 += 32 * WIN) {
-    uint32_t got[WIN];
-#pragma unroll
-    for (int w = 0; w < WIN; ++w) {
-      const long long i = i0 + 32 * w + lane;
-      got[w] = (i > row && i < p.n_rows) ? seg[i] : NO_SLOT;
-    }
+  // the other records of this slot, in row order; four 32-wide windows of rec_slot are in flight at once, and the
+  // compressed row of the next record is requested before the current one is merged
+  while (applied < pending && i0 < p.n_rows) {
 #pragma unroll
     for (int w = 0; w < WIN; ++w) {
       unsigned hits = __ballot_sync(FULL, got[w] == slot);
+      if (hits) load_fresh(p, i0 + 32 * w + __ffs(hits) - 1, lane, fid, fp);
       while (hits) {
-        const int j = __ffs(hits) - 1;
         hits &= hits - 1;
-        const long long i = i0 + 32 * w + j;
-        merge_warp(img, p.rec_ids + i * p.K, p.rec_p + i * p.K, p.K, lane);
+        const int cfid = fid;
+        const float cfp = fp;
+        if (hits) load_fresh(p, i0 + 32 * w + __ffs(hits) - 1, lane, fid, fp);
+        merge_warp(img, cfid, cfp, p.K, lane);
         ++applied;
       }
     }
+    i0 += 32 * WIN;
+    if (applied < pending && i0 < p.n_rows) {
+#pragma unroll
+      for (int w = 0; w < WIN; ++w) {
+        const long long i = i0 + 32 * w + lane;
+        got[w] = i < p.n_rows ? seg[i] : NO_SLOT;
+      }
+    }
   }
+  // the slot goes back as one line: update fields closed, entries past n_items zeroed
   const int n_items = (int)img->n_items;
-  if (lane < KMAX) {
-    s->ids[lane] = lane < n_items ? img->ids[lane] : 0;
-    s->probs[lane] = lane < n_items ? img->probs[lane] : 0.0f;
-  }
+  uint32_t out = word;  // key words unchanged
+  if (lane == 4) out = img->count;
+  if (lane == 5) out = img->n_items;
+  if (lane == 6) out = NO_REC;
+  if (lane == 7) out = 0u;
+  if (lane >= 8 && lane < 8 + KMAX) out = lane - 8 < n_items ? (uint32_t)img->ids[lane - 8] : 0u;
+  if (lane >= 8 + KMAX) out = lane - 8 - KMAX < n_items ? __float_as_uint(img->probs[lane - 8 - KMAX]) : 0u;
+  line[lane] = out;
   if (lane == 0) {
-    s->count = img->count;
-    s->n_items = img->n_items;
-    s->lead = NO_REC;
-    s->pend = 0;
     atomicAdd(&p.stats[ST_RECORDS], (unsigned long long)applied);
     if (fresh_slot) atomicAdd(&p.stats[ST_INSERTS], 1ull);
   }
