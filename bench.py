@@ -186,6 +186,9 @@ def run_ours(args, rank, world, local):
     torch.cuda.set_device(dev)
     dist = sd.init("nccl", dev)
     seed = sd.replica_seed(args.seed, rank)  # every rank runs its own sequences: independent replicas
+    # --sharded: one N-gram module for the sequences of all ranks; the ranks share the seed of the method's random
+    # numbers (counters tell the sequences apart) and start from the same table
+    lib_seed = args.seed if args.sharded else seed
     parent = inputs.topology(w.N, w.D, w.kb)
     depth = inputs.node_depths(parent)
     esize = 2 if w.dtype == inputs.DTYPE_BF16 else 4
@@ -197,9 +200,14 @@ def run_ours(args, rank, world, local):
     if args.ring:
         ring_n = args.ring
 
-    gpu = Stand(w.B, w.N, w.V, w.topk, w.order_max, w.dtype, w.T, seed, w.table_slots, parent, device=dev,
-                host_staging=True, deterministic=args.deterministic)
-    contexts = pregrow(gpu, w, seed, torch)
+    gpu = Stand(w.B, w.N, w.V, w.topk, w.order_max, w.dtype, w.T, lib_seed, w.table_slots, parent, device=dev,
+                host_staging=True, deterministic=args.deterministic, seq_base=rank * w.B if args.sharded else 0)
+    contexts = pregrow(gpu, w, lib_seed, torch)
+    if args.sharded:
+        from paper_2506_04708_b200 import sharded
+        step_fn = sharded.ShardedStand(gpu, dist).step
+    else:
+        step_fn = gpu.step
     prompt = 8
     streams = inputs.token_streams(w, seed, prompt + (ring_n + 4) * (w.D + 2))
     tail = np.full((w.B, w.order_max), -1, np.int32)
@@ -214,11 +222,11 @@ def run_ours(args, rank, world, local):
     for s in range(ring_n):
         gpu.lens_device(lens)
         gen.make(ring[s], lens, s)
-        gpu.step(ring[s])
+        step_fn(ring[s])
     del gen
     torch.cuda.empty_cache()
     for s in range(max(args.warmup, 3)):
-        gpu.step(ring[s % ring_n])
+        step_fn(ring[s % ring_n])
     torch.cuda.synchronize()
 
     def barrier():
@@ -237,7 +245,7 @@ def run_ours(args, rank, world, local):
     torch.cuda.nvtx.range_push("stand_timed")
     ev0.record()
     for s in range(args.steps):
-        gpu.step(ring[s % ring_n])
+        step_fn(ring[s % ring_n])
     ev1.record()
     barrier()
     torch.cuda.nvtx.range_pop()
@@ -254,23 +262,23 @@ def run_ours(args, rank, world, local):
         b.record()
     for s in range(n_prof):
         gpu.profile_row_pass(*evs[s])
-        gpu.step(ring[s % ring_n])
+        step_fn(ring[s % ring_n])
     gpu.profile_row_pass(None, None)
     torch.cuda.synchronize()
     k1_ms = statistics.mean(a.elapsed_time(b) for a, b in evs)
     # the same steps with events at every stage boundary (diagnostic: where the rest of a step goes)
-    n_st = min(args.steps, 100)
+    n_st = 0 if args.sharded else min(args.steps, 100)  # the stage events belong to the fused step
     sev = [[torch.cuda.Event(enable_timing=True) for _ in range(5)] for _ in range(n_st)]
     for row in sev:
         for e in row:
             e.record()
     for s in range(n_st):
         gpu.profile_stages(sev[s])
-        gpu.step(ring[s % ring_n])
+        step_fn(ring[s % ring_n])
     gpu.profile_stages(None)
     torch.cuda.synchronize()
-    stage_us = {name: 1e3 * statistics.mean(row[i].elapsed_time(row[i + 1]) for row in sev)
-                for i, name in enumerate(("row_pass", "verify", "update", "draft"))}
+    stage_us = None if not sev else {name: 1e3 * statistics.mean(row[i].elapsed_time(row[i + 1]) for row in sev)
+                                     for i, name in enumerate(("row_pass", "verify", "update", "draft"))}
     clocks = sampler.stop()
 
     ms_total = sd.max_over_ranks(dist, ms_total, dev)
@@ -285,11 +293,22 @@ def run_ours(args, rank, world, local):
     h_em = torch.empty((w.B, gpu.D + 1), dtype=torch.int32).pin_memory()
     h_ne = torch.empty(w.B, dtype=torch.int32).pin_memory()
     h_tr = torch.empty((w.B, w.N), dtype=torch.int32).pin_memory()
-    gpu.step_host(h_logits, h_em, h_ne, h_tr)
+    def host_step():
+        if not args.sharded:
+            gpu.step_host(h_logits, h_em, h_ne, h_tr)
+            return
+        ring[0].copy_(h_logits, non_blocking=True)
+        step_fn(ring[0])
+        h_em.copy_(gpu.emitted, non_blocking=True)
+        h_ne.copy_(gpu.n_emitted, non_blocking=True)
+        h_tr.copy_(gpu.tree, non_blocking=True)
+        torch.cuda.current_stream().synchronize()
+
+    host_step()
     barrier()
     t0 = time.perf_counter()
     for _ in range(e2e_steps):
-        gpu.step_host(h_logits, h_em, h_ne, h_tr)
+        host_step()
     barrier()
     e2e_s = time.perf_counter() - t0
     e2e_s = sd.max_over_ranks(dist, e2e_s, dev)
@@ -332,8 +351,8 @@ def run_ours(args, rank, world, local):
                        "drafting": "deterministic" if args.deterministic else "stochastic (Gumbel-Top-K)",
                        "l2": f"inputs larger than L2: {step_bytes / 1e6:.0f} MB per step, ring of {ring_n} "
                              f"buffers = {ring_n * step_bytes / 1e9:.2f} GB",
-                       "table_contexts_at_start": int(contexts), "multi_gpu": "independent replicas per GPU"
-                       if world > 1 else "single GPU", "acceptance_length": accept_len},
+                       "table_contexts_at_start": int(contexts), "multi_gpu": ("sequences sharded over the GPUs, one N-gram module: accepted rows all-gathered every step"
+                                     if args.sharded else "independent replicas per GPU" if world > 1 else "single GPU"), "acceptance_length": accept_len},
             "clocks": clocks, "e2e": e2e, "gpu_launches": int(launches), "roofline": roofline,
             "logits_gbs": alg_bytes * world / (ms_per_step * 1e-3) / 1e9,
             "stage_us": stage_us,
@@ -423,6 +442,9 @@ def main():
     ap.add_argument("--seed", type=int, default=0)
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--deterministic", action="store_true", help="deterministic drafting (paper Sec. 3.2) instead of stochastic")
+    ap.add_argument("--sharded", action="store_true",
+                    help="one N-gram module shared by the sequences of all ranks (accepted rows exchanged every step) "
+                         "instead of independent replicas")
     ap.add_argument("--no-sweep", action="store_true", help="skip the short runs of the other four workloads")
     ap.add_argument("--batch", type=int, default=0, help="override the workload's number of sequences (profiling)")
     ap.add_argument("--ring", type=int, default=0, help="override the number of logit buffers in the ring (profiling)")

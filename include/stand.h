@@ -71,6 +71,9 @@ typedef struct {
   int32_t deterministic;   /* 0: stochastic drafting (Sec. 4.2); 1: deterministic drafting (Sec. 3.2): the children of a
                               node are its most probable candidates in order, each verified as a one-hot draft */
   int32_t host_staging;    /* != 0: reserve a logits staging buffer for stand_step_host */
+  int32_t seq_base;        /* global index of this context's sequence 0, >= 0.  The random-number counters use
+                              seq_base + b, so a batch split over several contexts draws what the whole batch would */
+  int32_t reserved;        /* must be 0 */
 } stand_config;
 
 typedef struct {
@@ -129,6 +132,19 @@ int stand_ngram_update(stand_ctx* ctx, void* cu_stream);
  * applied in row order, each under every order it is long enough for. */
 int stand_ngram_update_bulk(stand_ctx* ctx, const int32_t* dev_ctx, const int32_t* dev_ids, const float* dev_probs,
                             int64_t M, void* cu_stream);
+
+/* Sec. 4.1 when the sequences of one N-gram module are split over several contexts (one per GPU): the
+ * accepted rows of the last verification in the layout stand_ngram_update_bulk takes.  Writes B * (D+1)
+ * rows in (sequence, path position) order: dev_ctx [B*(D+1), order_max], dev_ids / dev_probs
+ * [B*(D+1), topk].  Positions past a sequence's accepted path get an all -1 context, ids -1 and
+ * probabilities 0; a bulk update skips them.  Every context then applies the rows of all contexts,
+ * concatenated in the order of their seq_base, with stand_ngram_update_bulk: each table ends up as the
+ * table of one context that held all the sequences.  STAND_E_STATE without a pending verification. */
+int stand_export_records(stand_ctx* ctx, int32_t* dev_ctx, int32_t* dev_ids, float* dev_probs, void* cu_stream);
+
+/* Drops the pending verification's own update (its rows reach the tables through
+ * stand_ngram_update_bulk instead).  Host only.  STAND_E_STATE if no verification is pending. */
+int stand_skip_update(stand_ctx* ctx);
 
 /* Sec. 4.2: drafts the next tree of every sequence.  Breadth-first over the static
  * topology; for a node with children the contexts of order order_max..1 are looked

@@ -17,7 +17,7 @@ DTYPE_F32, DTYPE_BF16 = 0, 1
 
 EXPORTS = [
     "stand_workspace_bytes", "stand_init", "stand_destroy", "stand_reset_sequences", "stand_verify_tree",
-    "stand_ngram_update", "stand_ngram_update_bulk", "stand_draft_tree", "stand_step", "stand_step_host",
+    "stand_ngram_update", "stand_ngram_update_bulk", "stand_export_records", "stand_skip_update", "stand_draft_tree", "stand_step", "stand_step_host",
     "stand_row_stats_scratch_bytes", "stand_row_stats", "stand_row_stats_static", "stand_get_stats",
     "stand_last_path", "stand_tree_depth", "stand_table_dump", "stand_table_load", "stand_state_dump",
     "stand_state_load", "stand_profile_row_pass", "stand_profile_stages", "stand_node_accepts", "stand_prune_tree",
@@ -30,7 +30,7 @@ class StandConfig(C.Structure):
         ("B", C.c_int32), ("N", C.c_int32), ("V", C.c_int32), ("topk", C.c_int32), ("order_max", C.c_int32),
         ("dtype", C.c_int32), ("temperature", C.c_float), ("max_probe", C.c_int32), ("seed", C.c_uint64),
         ("table_slots", C.c_uint64), ("parent", C.c_void_p), ("deterministic", C.c_int32),
-        ("host_staging", C.c_int32),
+        ("host_staging", C.c_int32), ("seq_base", C.c_int32), ("reserved", C.c_int32),
     ]
 
 
@@ -67,6 +67,10 @@ def lib():
     L.stand_verify_tree.argtypes = [vp, vp, vp, vp, vp]
     L.stand_ngram_update.argtypes = [vp, vp]
     L.stand_ngram_update_bulk.argtypes = [vp, vp, vp, vp, i64, vp]
+    L.stand_export_records.argtypes = [vp, vp, vp, vp, vp]
+    L.stand_export_records.restype = C.c_int
+    L.stand_skip_update.argtypes = [vp]
+    L.stand_skip_update.restype = C.c_int
     L.stand_draft_tree.argtypes = [vp, vp, vp]
     L.stand_step.argtypes = [vp, vp, vp, vp, vp, vp]
     L.stand_step_host.argtypes = [vp, vp, vp, vp, vp, vp]
@@ -122,10 +126,10 @@ def _stream(stream):
 
 
 def make_config(B, N, V, topk, order_max, dtype, temperature, seed, table_slots, parent, max_probe=0,
-                host_staging=False, deterministic=False):
+                host_staging=False, deterministic=False, seq_base=0):
     par = np.ascontiguousarray(parent, np.int32)
     cfg = StandConfig(B, N, V, topk, order_max, dtype, float(temperature), max_probe, seed, table_slots,
-                      par.ctypes.data, int(bool(deterministic)), int(bool(host_staging)))
+                      par.ctypes.data, int(bool(deterministic)), int(bool(host_staging)), int(seq_base), 0)
     cfg._keepalive = par
     return cfg
 
@@ -138,13 +142,15 @@ class Stand:
     """One decoder context.  Tensors are torch CUDA tensors; results are written in place."""
 
     def __init__(self, B, N, V, topk, order_max, dtype, temperature, seed, table_slots, parent, max_probe=0,
-                 host_staging=False, device="cuda:0", deterministic=False):
+                 host_staging=False, device="cuda:0", deterministic=False, seq_base=0):
         import torch
         self.torch = torch
         self.dev = torch.device(device)
         self.B, self.N, self.V, self.K, self.n_max, self.dtype = B, N, V, topk, order_max, dtype
         self.cfg = make_config(B, N, V, topk, order_max, dtype, temperature, seed, table_slots, parent, max_probe,
-                               host_staging, deterministic)
+                               host_staging, deterministic, seq_base)
+        self.seq_base = seq_base
+        self._bulk_keep = None
         need = workspace_bytes(self.cfg)
         if need == 0:
             raise StandError("invalid configuration")
@@ -192,7 +198,9 @@ class Stand:
     def ngram_update(self, stream=None):
         _check(lib().stand_ngram_update(self.h, _stream(stream)), "stand_ngram_update")
 
-    def ngram_update_bulk(self, ctx, ids, probs, stream=None):
+    def ngram_update_bulk(self, ctx, ids, probs, stream=None, sync=True):
+        """Rows [M, order_max] / [M, topk] / [M, topk].  sync=False returns without waiting for the kernels
+        and keeps the three tensors alive until the next bulk update."""
         t = self.torch
         ctx = ctx.to(device=self.dev, dtype=t.int32).contiguous()
         ids = ids.to(device=self.dev, dtype=t.int32).contiguous()
@@ -201,7 +209,26 @@ class Stand:
         assert ids.numel() == M * self.K and probs.numel() == M * self.K
         _check(lib().stand_ngram_update_bulk(self.h, _ptr(ctx), _ptr(ids), _ptr(probs), M, _stream(stream)),
                "stand_ngram_update_bulk")
-        (t.cuda.current_stream() if stream is None else stream).synchronize()  # inputs must outlive the kernels
+        if sync:
+            (t.cuda.current_stream() if stream is None else stream).synchronize()  # inputs must outlive the kernels
+            self._bulk_keep = None
+        else:
+            self._bulk_keep = (ctx, ids, probs)
+
+    def export_records(self, stream=None):
+        """The accepted rows of the last verification as bulk-update rows: (ctx [B*(D+1), order_max] int32,
+        ids [B*(D+1), topk] int32, probs [B*(D+1), topk] float32), device tensors; rows past a path are blank."""
+        t = self.torch
+        rows = self.B * (self.D + 1)
+        ctx = t.empty((rows, self.n_max), dtype=t.int32, device=self.dev)
+        ids = t.empty((rows, self.K), dtype=t.int32, device=self.dev)
+        probs = t.empty((rows, self.K), dtype=t.float32, device=self.dev)
+        _check(lib().stand_export_records(self.h, _ptr(ctx), _ptr(ids), _ptr(probs), _stream(stream)),
+               "stand_export_records")
+        return ctx, ids, probs
+
+    def skip_update(self):
+        _check(lib().stand_skip_update(self.h), "stand_skip_update")
 
     def draft_tree(self, stream=None):
         _check(lib().stand_draft_tree(self.h, _ptr(self.tree), _stream(stream)), "stand_draft_tree")

@@ -34,6 +34,7 @@ struct DraftParams {
   float* cand_phi;         // [B, N, K]
   unsigned long long* stats;
   int deterministic;       // != 0: the children are the most probable candidates, no noise
+  int seq_base;            // global index of sequence 0 (random-number counters use seq_base + b)
 };
 
 // Rank of this lane's candidate by g = log(phi) - log(-log U) in double precision (larger first, equal
@@ -135,7 +136,7 @@ __global__ void __launch_bounds__(K4_THREADS) draft_kernel(const DraftParams p) 
       // Perturbed scores in single precision first; they decide the order whenever every pair of
       // candidates is further apart than single precision can blur (1e-3 against errors of a few 1e-6).
       // Otherwise the scores are formed again in double precision.
-      const uint32_t u24 = (valid && !p.deterministic) ? philox_u24(p.seed, b, p.step, u, SLOT_GUMBEL | (uint32_t)id) : 0u;
+      const uint32_t u24 = (valid && !p.deterministic) ? philox_u24(p.seed, (uint32_t)(p.seq_base + b), p.step, u, SLOT_GUMBEL | (uint32_t)id) : 0u;
       float gf = 0.0f;
       if (valid && p.deterministic) gf = phi;  // deterministic drafting (Sec. 3.2): rank by the stored probability itself
       else if (valid) {

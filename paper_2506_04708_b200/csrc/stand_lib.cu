@@ -39,6 +39,7 @@ bool derive(const stand_config* c, Derived* d) {
   if (c->topk < 1 || c->topk > STAND_MAX_TOPK || c->order_max < 1 || c->order_max > STAND_MAX_ORDER) return false;
   if (c->dtype != STAND_DTYPE_F32 && c->dtype != STAND_DTYPE_BF16) return false;
   if (!(c->temperature > 0.0f) || c->max_probe < 0 || (c->deterministic != 0 && c->deterministic != 1)) return false;
+  if (c->seq_base < 0 || (long long)c->seq_base + c->B > 0x7FFFFFFFll || c->reserved != 0) return false;
   if (c->table_slots < 2 || (c->table_slots & (c->table_slots - 1)) != 0 || c->table_slots > (1ull << 32) - 2) return false;
   if (!c->parent || c->parent[0] != -1) return false;
   if ((long long)c->B * c->N > (1ll << 31) / 4) return false;
@@ -257,6 +258,7 @@ int run_verify(stand_ctx* x, const void* logits, int32_t* emitted, int32_t* n_em
   v.stats = x->at<unsigned long long>(x->L.stats);
   v.node_accepts = x->at<unsigned long long>(x->L.accepts);
   v.deterministic = c.deterministic;
+  v.seq_base = c.seq_base;
   v.fuse_locate = fuse_locate ? 1 : 0;
   v.upd = step_update_params(x);
   // inside a fused step (and with no timing events between the launches) the kernels chain programmatically
@@ -306,6 +308,7 @@ int run_draft(stand_ctx* x, int32_t* tree_user, bool chained, cudaStream_t st) {
   d.tree_user = tree_user; d.cand_n = x->at<int>(x->L.cand_n); d.cand_id = x->at<int>(x->L.cand_id);
   d.cand_phi = x->at<float>(x->L.cand_phi); d.stats = x->at<unsigned long long>(x->L.stats);
   d.deterministic = c.deterministic;
+  d.seq_base = c.seq_base;
   int rc;
   if (chained && !x->ev_stage[3]) rc = launch_dependent(draft_kernel, (unsigned)c.B, K4_THREADS, st, d);
   else { draft_kernel<<<c.B, K4_THREADS, 0, st>>>(d); rc = launch_ok(); }
@@ -320,6 +323,24 @@ __global__ void reset_tree_kernel(int B, int N, int n_max, const int* tail, int*
   const int b = (int)(i / N), u = (int)(i % N);
   tree[i] = u == 0 ? tail[b * n_max + n_max - 1] : -1;
   cand_n[i] = 0;
+}
+
+// The records of the last verification as rows for a bulk update: positions past a sequence's accepted
+// path get an all -1 context (a bulk update skips such a row), ids -1 and probabilities 0.
+__global__ void export_records_kernel(int B, int W, int n_max, int K, const int* n_path, const int* rec_ctx, const int* rec_ids,
+                                      const float* rec_p, int* out_ctx, int* out_ids, float* out_p) {
+  const long long i = (long long)blockIdx.x * blockDim.x + threadIdx.x;  // one thread per (row, entry)
+  const int per_row = n_max + K;
+  if (i >= (long long)B * W * per_row) return;
+  const long long row = i / per_row;
+  const int e = (int)(i - row * per_row);
+  const bool live = (int)(row % W) < n_path[row / W];
+  if (e < n_max) out_ctx[row * n_max + e] = live ? rec_ctx[row * n_max + e] : -1;
+  else {
+    const int k = e - n_max;
+    out_ids[row * K + k] = live ? rec_ids[row * K + k] : -1;
+    out_p[row * K + k] = live ? rec_p[row * K + k] : 0.0f;
+  }
 }
 
 }  // namespace
@@ -441,6 +462,29 @@ int stand_ngram_update_bulk(stand_ctx* x, const int32_t* dev_ctx, const int32_t*
                                                     dev_probs + at * c.topk, nullptr, 1), false, st);
     if (rc) return rc;
   }
+  return STAND_OK;
+}
+
+int stand_export_records(stand_ctx* x, int32_t* dev_ctx, int32_t* dev_ids, float* dev_probs, void* cu_stream) {
+  if (!x || !dev_ctx || !dev_ids || !dev_probs) return STAND_E_ARG;
+  if (!x->pending) return STAND_E_STATE;
+  cudaStream_t st = (cudaStream_t)cu_stream;
+  x->last_stream = st;
+  const stand_config& c = x->cfg;
+  const int W = x->d.D + 1;
+  const long long n = (long long)c.B * W * (c.order_max + c.topk);
+  export_records_kernel<<<(unsigned)((n + 255) / 256), 256, 0, st>>>(c.B, W, c.order_max, c.topk, x->at<int>(x->L.n_path),
+                                                                     x->at<int>(x->L.rec_ctx), x->at<int>(x->L.rec_ids),
+                                                                     x->at<float>(x->L.rec_p), dev_ctx, dev_ids, dev_probs);
+  const int rc = launch_ok();
+  if (rc == STAND_OK) x->launches += 1;
+  return rc;
+}
+
+int stand_skip_update(stand_ctx* x) {
+  if (!x) return STAND_E_ARG;
+  if (!x->pending || x->located) return STAND_E_STATE;  // located: slots are already marked for the update
+  x->pending = false;
   return STAND_OK;
 }
 

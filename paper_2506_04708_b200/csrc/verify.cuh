@@ -53,6 +53,7 @@ struct VerifyParams {
   unsigned long long* stats;
   unsigned long long* node_accepts;  // [N] how often each node lay on an accepted path
   int deterministic;       // != 0: deterministic drafting (every drafted token is a one-hot draft)
+  int seq_base;            // global index of sequence 0 (random-number counters use seq_base + b)
   int fuse_locate;         // != 0: also run stage 1 of the N-gram update for this sequence's records
   UpdateParams upd;        // used when fuse_locate is set
 };
@@ -369,7 +370,7 @@ __global__ void __launch_bounds__(K2_THREADS, 2) verify_kernel(const VerifyParam
       double qh = li < nc ? (double)s_cphi[(u) * KMAX + (li)] : 0.0;
       double qn = half_sum_d(qh), zr = 1.0, pq = 1.0;
       // the uniforms of all children at once
-      const double Uj = li < drafted ? (double)philox_u24(p.seed, b, p.step, u, (uint32_t)li) * (1.0 / 16777216.0) : 0.0;
+      const double Uj = li < drafted ? (double)philox_u24(p.seed, (uint32_t)(p.seq_base + b), p.step, u, (uint32_t)li) * (1.0 / 16777216.0) : 0.0;
       int accepted = -1;
       for (int j = 0; j < drafted; ++j) {
         const int x = s_tree[fc + j];
@@ -425,7 +426,7 @@ __global__ void __launch_bounds__(K2_THREADS, 2) verify_kernel(const VerifyParam
   const double scale = s_scale;
   const float off = s_off[us];
   const double invZ = s_invZ[us];
-  const double U = (double)philox_u24(p.seed, b, p.step, us, SLOT_FINAL) * (1.0 / 16777216.0);
+  const double U = (double)philox_u24(p.seed, (uint32_t)(p.seq_base + b), p.step, us, SLOT_FINAL) * (1.0 / 16777216.0);
 
   // coarse: mass of every chunk; thread t owns `per` consecutive chunks
   const int per = (p.n_chunks + K2_THREADS - 1) / K2_THREADS;  // <= 4 for V <= 2^20

@@ -7,7 +7,7 @@ import sys
 import pytest
 import torch.multiprocessing as mp
 
-from paper_2506_04708_b200 import dist as sd, inputs
+from paper_2506_04708_b200 import dist as sd, inputs, sharded
 
 ROOT = os.path.dirname(os.path.dirname(os.path.abspath(__file__)))
 
@@ -57,3 +57,41 @@ def test_reference_arm_runs_on_rank_zero_only():
     out = subprocess.run([sys.executable, os.path.join(ROOT, "bench.py"), "--impl", "reference", "--gpus", "2", "--steps", "1",
                           "--warmup", "0"], env=env, capture_output=True, text=True, timeout=120)
     assert out.returncode == 0 and out.stdout.strip() == ""
+
+
+def _exchange_worker(rank, world, port, out_dir):
+    import numpy as np
+    import torch
+    os.environ.update(RANK=str(rank), WORLD_SIZE=str(world), LOCAL_RANK=str(rank), MASTER_ADDR="127.0.0.1",
+                      MASTER_PORT=str(port))
+    d = sd.init("gloo")
+    B, W, n_max, K = 3, 4, 3, 5  # sequences per rank, path slots per sequence
+    seq = rank * B + torch.arange(B).repeat_interleave(W)          # global sequence of every row
+    pos = torch.arange(W).repeat(B)
+    ctx = torch.stack([seq, pos, seq * 100 + pos], dim=1).to(torch.int32)
+    ids = (seq * 1000 + pos * 10).to(torch.int32)[:, None] + torch.arange(K, dtype=torch.int32)[None, :]
+    probs = (seq.double() + pos.double() / 10)[:, None].float().repeat(1, K)
+    g_ctx, g_ids, g_probs = sharded.gather_rows(d, (ctx, ids, probs))
+    np.savez(os.path.join(out_dir, f"x{rank}.npz"), ctx=g_ctx.numpy(), ids=g_ids.numpy(), probs=g_probs.numpy())
+    sd.barrier(d)
+    d.destroy_process_group()
+
+
+def test_record_exchange_keeps_global_sequence_order(tmp_path):
+    """The update rows of all ranks arrive on every rank in (sequence, path position) order of the whole batch: the
+    order in which one context holding the whole batch applies them."""
+    import numpy as np
+    world, port = 2, 31000 + os.getpid() % 2000
+    mp.spawn(_exchange_worker, args=(world, port, str(tmp_path)), nprocs=world, join=True)
+    r = [np.load(tmp_path / f"x{k}.npz") for k in range(world)]
+    for k in ("ctx", "ids", "probs"):
+        assert np.array_equal(r[0][k], r[1][k])
+    ctx = r[0]["ctx"]
+    assert ctx.shape == (2 * 3 * 4, 3)
+    order = ctx[:, 0] * 4 + ctx[:, 1]
+    assert np.array_equal(order, np.arange(24))
+    assert np.array_equal(r[0]["ids"][:, 0], ctx[:, 0] * 1000 + ctx[:, 1] * 10)
+    # no group: the rows pass through untouched
+    import torch
+    rows = (torch.zeros(2, 3), torch.zeros(2, 5), torch.zeros(2, 5))
+    assert sharded.gather_rows(None, rows) is rows

@@ -338,6 +338,55 @@ def test_stage_calls_equal_the_fused_step():
     a.close(); b.close()
 
 
+@pytest.mark.parametrize("deterministic", [False, True])
+def test_sharded_contexts_equal_the_unsharded_one(deterministic):
+    """A batch of 6 sequences split 2 + 4 over two contexts (seq_base 0 and 2), each with its own copy of the
+    table, the accepted rows exchanged every step and applied in global sequence order: emitted tokens, drafts
+    and both tables equal those of one context holding all 6 (which the other tests tie to the oracle)."""
+    torch = _torch()
+    from paper_2506_04708_b200.binding import Stand, StandError
+    from paper_2506_04708_b200 import sharded
+    w = inputs.scaled(inputs.WORKLOADS["cfg1"], B=6, steps=40)
+    parent = inputs.topology(w.N, w.D, w.kb)
+    depth = inputs.node_depths(parent)
+    streams = inputs.token_streams(w, 5, 500)
+    mk = lambda B, base: Stand(B, w.N, w.V, w.topk, w.order_max, w.dtype, w.T, 5, 1 << 14, parent,
+                               deterministic=deterministic, seq_base=base)
+    whole = mk(6, 0)
+    cuts = [(0, 2), (2, 6)]
+    parts = [sharded.ShardedStand(mk(hi - lo, lo)) for lo, hi in cuts]
+    tail = torch.from_numpy(streams[:, 5:8].copy())
+    lens = np.full(w.B, 8, np.int64)
+    whole.reset_sequences(tail, torch.from_numpy(lens))
+    for (lo, hi), sh in zip(cuts, parts):
+        sh.stand.reset_sequences(tail[lo:hi], torch.from_numpy(lens[lo:hi]))
+    for s in range(40):
+        dl = harness.to_device_logits(inputs.logits_numpy(w, streams, lens, depth, s, 5, "p80"))
+        ew, nw, tw = (t.cpu().numpy().copy() for t in whole.step(dl))
+        rows = [sh.verify(dl[lo:hi].contiguous()) for (lo, hi), sh in zip(cuts, parts)]
+        all_rows = sharded.concat_rows(rows)
+        for (lo, hi), sh in zip(cuts, parts):
+            tree = sh.finish(all_rows)
+            assert np.array_equal(ew[lo:hi], sh.stand.emitted.cpu().numpy()), s
+            assert np.array_equal(nw[lo:hi], sh.stand.n_emitted.cpu().numpy()), s
+            assert np.array_equal(tw[lo:hi], tree.cpu().numpy()), s
+        lens = whole.state_dump()["len"]
+    assert nw.sum() > w.B  # drafts were accepted: the tables matter
+    t0 = whole.table_dict()
+    assert len(t0) > 100
+    for sh in parts:
+        assert sh.stand.table_dict() == t0
+        assert sh.stand.stats()["drops"] == 0
+    # nothing pending any more: neither export nor skip is valid
+    with pytest.raises(StandError):
+        parts[0].stand.export_records()
+    with pytest.raises(StandError):
+        parts[0].stand.skip_update()
+    whole.close()
+    for sh in parts:
+        sh.stand.close()
+
+
 def test_table_persists_across_trajectories_and_resume_from_a_checkpoint():
     """Sec. 5.1: the N-gram module is kept across trajectories (stand_reset_sequences restarts the sequences only).
     And a run resumed in a fresh context from dumped table + state continues exactly like the original."""
