@@ -119,9 +119,9 @@ def workload_of(args):
 
 
 # DRAM bytes per row-pass launch from the ncu capture summarised in profiles/row_pass_kernel_cfg5_B64_ncu_full.md
-# (dram__bytes_read.sum + dram__bytes_write.sum = 466.77 MB + 7.8 MB at B=64; traffic grows with the rows, so a
+# (dram__bytes_read.sum + dram__bytes_write.sum = 466.79 MB + 3.6 MB at B=64; traffic grows with the rows, so a
 # launch over B sequences moves B/64 times that).  None for shapes that were not captured.
-ROW_PASS_TRAFFIC_PER_SEQUENCE = {"cfg5": (466.77e6 + 7.8e6) / 64}
+ROW_PASS_TRAFFIC_PER_SEQUENCE = {"cfg5": (466.79e6 + 3.6e6) / 64}
 
 
 def quick_workload(name, args, dev, peaks):
