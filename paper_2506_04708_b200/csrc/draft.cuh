@@ -55,13 +55,16 @@ __device__ __noinline__ int gumbel_rank_double(bool valid, int id, float phi, ui
   return rank;
 }
 
-__global__ void __launch_bounds__(K4_THREADS) draft_kernel(const DraftParams p) {
+// The next tree of sequence b by one block of K4_THREADS threads.  WAIT: stop (griddepcontrol.wait) before the first
+// read of what the previous kernel wrote; false when the caller has already ordered itself after that kernel.
+template <bool WAIT>
+__device__ __forceinline__ void draft_block(const DraftParams& p, const int b) {
   __shared__ int s_tok[NODES_MAX], s_parent[NODES_MAX], s_fc[NODES_MAX], s_nch[NODES_MAX];
   __shared__ int s_tail[ORDER_MAX], s_level[DEPTH_MAX + 2];
   __shared__ Slot s_slot[K4_THREADS / 32];  // per warp: the slot that won the lookup
   __shared__ float s_g[K4_THREADS / 32][KMAX];  // per warp: the candidates' perturbed scores and ids
   __shared__ int s_gid[K4_THREADS / 32][KMAX];
-  const int b = blockIdx.x, tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+  const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
   const int N = p.N, K = p.K, n_max = p.n_max;
   pdl_trigger();
   // topology and tail once, with coalesced loads: the level loop below touches shared memory only
@@ -72,7 +75,7 @@ __global__ void __launch_bounds__(K4_THREADS) draft_kernel(const DraftParams p) 
     s_nch[u] = p.n_children[u];
   }
   if (tid <= p.D + 1) s_level[tid] = p.level_start[tid];
-  pdl_wait();  // tails come from the verification, the table from the update
+  if (WAIT) pdl_wait();  // tails come from the verification, the table from the update
   if (tid < n_max) s_tail[tid] = p.tail[b * n_max + tid];
   __syncthreads();
   if (tid == 0) s_tok[0] = s_tail[n_max - 1];  // the root carries the last token
@@ -185,5 +188,7 @@ __global__ void __launch_bounds__(K4_THREADS) draft_kernel(const DraftParams p) 
     if (p.tree_user) p.tree_user[(long long)b * N + u] = t;
   }
 }
+
+__global__ void __launch_bounds__(K4_THREADS) draft_kernel(const DraftParams p) { draft_block<true>(p, (int)blockIdx.x); }
 
 }  // namespace stand

@@ -13,6 +13,7 @@
 #include "draft.cuh"
 #include "row_pass.cuh"
 #include "table.cuh"
+#include "tail.cuh"
 #include "verify.cuh"
 
 using namespace stand;
@@ -160,6 +161,9 @@ int prepare_device(int* sm_count) {
     if (cudaFuncSetAttribute(verify_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)verify_smem_bytes(NODES_MAX)) !=
         cudaSuccess)
       return STAND_E_CUDA;
+    if (cudaFuncSetAttribute(tail_single_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)verify_smem_bytes(NODES_MAX)) !=
+        cudaSuccess)
+      return STAND_E_CUDA;
     g_sm_count[dev].store(sms, std::memory_order_relaxed);
     g_k1_ready[dev].store(1, std::memory_order_release);
   }
@@ -233,18 +237,8 @@ UpdateParams step_update_params(stand_ctx* x) {
                        x->at<float>(x->L.rec_p), x->at<int>(x->L.n_path), W);
 }
 
-// fuse_locate: the verification kernel also maps this step's records to table slots (stage 1 of the update).
-int run_verify(stand_ctx* x, const void* logits, int32_t* emitted, int32_t* n_emitted, bool fuse_locate, cudaStream_t st) {
+VerifyParams verify_params(stand_ctx* x, const void* logits, int32_t* emitted, int32_t* n_emitted, bool fuse_locate) {
   const stand_config& c = x->cfg;
-  if (x->ev_before) cudaEventRecord(x->ev_before, st);
-  if (x->ev_stage[0]) cudaEventRecord(x->ev_stage[0], st);
-  int rc = launch_row_pass(logits, (long long)c.B * c.N, c.V, c.dtype, x->d.n_chunks, x->c, x->at<float2>(x->L.pairs),
-                           x->at<int>(x->L.status), st, fuse_locate && !x->ev_before && !x->ev_stage[0]);
-  if (rc) return rc;
-  if (x->ev_after) cudaEventRecord(x->ev_after, st);
-  if (x->ev_stage[1]) cudaEventRecord(x->ev_stage[1], st);
-  x->launches += 1;
-  x->step += 1;  // the tree drafted in step s-1 is verified in step s
   VerifyParams v;
   v.logits = logits; v.dtype = c.dtype; v.B = c.B; v.N = c.N; v.V = c.V; v.K = c.topk; v.n_max = c.order_max;
   v.D = x->d.D; v.n_chunks = x->d.n_chunks; v.c = x->c; v.seed = c.seed; v.step = x->step;
@@ -261,6 +255,36 @@ int run_verify(stand_ctx* x, const void* logits, int32_t* emitted, int32_t* n_em
   v.seq_base = c.seq_base;
   v.fuse_locate = fuse_locate ? 1 : 0;
   v.upd = step_update_params(x);
+  return v;
+}
+
+DraftParams draft_params(stand_ctx* x, int32_t* tree_user) {
+  const stand_config& c = x->cfg;
+  DraftParams d;
+  d.table = x->at<Slot>(x->L.table); d.mask = c.table_slots - 1; d.max_probe = x->max_probe; d.B = c.B; d.N = c.N;
+  d.K = c.topk; d.n_max = c.order_max; d.D = x->d.D; d.V = c.V; d.seed = c.seed; d.step = x->step;
+  d.parent = x->topo_parent(); d.first_child = x->topo_first_child(); d.n_children = x->topo_n_children();
+  d.level_start = x->topo_level_start(); d.tail = x->at<int>(x->L.tail); d.tree = x->at<int>(x->L.tree);
+  d.tree_user = tree_user; d.cand_n = x->at<int>(x->L.cand_n); d.cand_id = x->at<int>(x->L.cand_id);
+  d.cand_phi = x->at<float>(x->L.cand_phi); d.stats = x->at<unsigned long long>(x->L.stats);
+  d.deterministic = c.deterministic;
+  d.seq_base = c.seq_base;
+  return d;
+}
+
+// fuse_locate: the verification kernel also maps this step's records to table slots (stage 1 of the update).
+int run_verify(stand_ctx* x, const void* logits, int32_t* emitted, int32_t* n_emitted, bool fuse_locate, cudaStream_t st) {
+  const stand_config& c = x->cfg;
+  if (x->ev_before) cudaEventRecord(x->ev_before, st);
+  if (x->ev_stage[0]) cudaEventRecord(x->ev_stage[0], st);
+  int rc = launch_row_pass(logits, (long long)c.B * c.N, c.V, c.dtype, x->d.n_chunks, x->c, x->at<float2>(x->L.pairs),
+                           x->at<int>(x->L.status), st, fuse_locate && !x->ev_before && !x->ev_stage[0]);
+  if (rc) return rc;
+  if (x->ev_after) cudaEventRecord(x->ev_after, st);
+  if (x->ev_stage[1]) cudaEventRecord(x->ev_stage[1], st);
+  x->launches += 1;
+  x->step += 1;  // the tree drafted in step s-1 is verified in step s
+  const VerifyParams v = verify_params(x, logits, emitted, n_emitted, fuse_locate);
   // inside a fused step (and with no timing events between the launches) the kernels chain programmatically
   const bool chain = fuse_locate && !x->ev_after && !x->ev_stage[1];
   const size_t vsm = verify_smem_bytes(c.N);
@@ -300,21 +324,46 @@ int run_update(stand_ctx* x, cudaStream_t st) {
 
 int run_draft(stand_ctx* x, int32_t* tree_user, bool chained, cudaStream_t st) {
   const stand_config& c = x->cfg;
-  DraftParams d;
-  d.table = x->at<Slot>(x->L.table); d.mask = c.table_slots - 1; d.max_probe = x->max_probe; d.B = c.B; d.N = c.N;
-  d.K = c.topk; d.n_max = c.order_max; d.D = x->d.D; d.V = c.V; d.seed = c.seed; d.step = x->step;
-  d.parent = x->topo_parent(); d.first_child = x->topo_first_child(); d.n_children = x->topo_n_children();
-  d.level_start = x->topo_level_start(); d.tail = x->at<int>(x->L.tail); d.tree = x->at<int>(x->L.tree);
-  d.tree_user = tree_user; d.cand_n = x->at<int>(x->L.cand_n); d.cand_id = x->at<int>(x->L.cand_id);
-  d.cand_phi = x->at<float>(x->L.cand_phi); d.stats = x->at<unsigned long long>(x->L.stats);
-  d.deterministic = c.deterministic;
-  d.seq_base = c.seq_base;
+  const DraftParams d = draft_params(x, tree_user);
   int rc;
   if (chained && !x->ev_stage[3]) rc = launch_dependent(draft_kernel, (unsigned)c.B, K4_THREADS, st, d);
   else { draft_kernel<<<c.B, K4_THREADS, 0, st>>>(d); rc = launch_ok(); }
   if (rc == STAND_OK) x->launches += 1;
   if (x->ev_stage[4]) cudaEventRecord(x->ev_stage[4], st);
   return rc;
+}
+
+bool timing_hooks(const stand_ctx* x) {
+  if (x->ev_before || x->ev_after) return true;
+  for (int i = 0; i < 5; ++i)
+    if (x->ev_stage[i]) return true;
+  return false;
+}
+
+// One whole step on a stream.  A single sequence takes two launches (row pass, then its whole tail in one
+// block); batches take four.
+int run_step(stand_ctx* x, const void* logits, int32_t* emitted, int32_t* n_emitted, int32_t* tree_user, cudaStream_t st) {
+  const stand_config& c = x->cfg;
+  if (c.B == 1 && !timing_hooks(x)) {
+    int rc = launch_row_pass(logits, (long long)c.N, c.V, c.dtype, x->d.n_chunks, x->c, x->at<float2>(x->L.pairs),
+                             x->at<int>(x->L.status), st, true);
+    if (rc) return rc;
+    x->step += 1;
+    TailParams t;
+    t.v = verify_params(x, logits, emitted, n_emitted, true);
+    t.d = draft_params(x, tree_user);
+    rc = launch_dependent(tail_single_kernel, 1u, K2_THREADS, st, t, verify_smem_bytes(c.N));
+    if (rc) return rc;
+    x->launches += 2;
+    x->pending = false;
+    x->located = false;
+    return STAND_OK;
+  }
+  int rc = run_verify(x, logits, emitted, n_emitted, true, st);
+  if (rc) return rc;
+  rc = run_update(x, st);
+  if (rc) return rc;
+  return run_draft(x, tree_user, true, st);
 }
 
 __global__ void reset_tree_kernel(int B, int N, int n_max, const int* tail, int* tree, int* cand_n) {
@@ -500,11 +549,7 @@ int stand_step(stand_ctx* x, const void* dev_logits, int32_t* dev_emitted, int32
   cudaStream_t st = (cudaStream_t)cu_stream;
   x->last_stream = st;
   if (x->pending && x->located) return STAND_E_STATE;
-  int rc = run_verify(x, dev_logits, dev_emitted, dev_n_emitted, true, st);
-  if (rc) return rc;
-  rc = run_update(x, st);
-  if (rc) return rc;
-  return run_draft(x, dev_tree_tokens, true, st);
+  return run_step(x, dev_logits, dev_emitted, dev_n_emitted, dev_tree_tokens, st);
 }
 
 int stand_step_host(stand_ctx* x, const void* host_logits, int32_t* host_emitted, int32_t* host_n_emitted,
@@ -517,11 +562,7 @@ int stand_step_host(stand_ctx* x, const void* host_logits, int32_t* host_emitted
   const size_t bytes = (size_t)c.B * c.N * c.V * esize_of(c.dtype);
   int rc = cuda_ok(cudaMemcpyAsync(x->ws + x->L.staging, host_logits, bytes, cudaMemcpyHostToDevice, st));
   if (rc) return rc;
-  rc = run_verify(x, x->ws + x->L.staging, nullptr, nullptr, true, st);
-  if (rc) return rc;
-  rc = run_update(x, st);
-  if (rc) return rc;
-  rc = run_draft(x, nullptr, true, st);
+  rc = run_step(x, x->ws + x->L.staging, nullptr, nullptr, nullptr, st);
   if (rc) return rc;
   const size_t W = x->d.D + 1;
   if (host_emitted) rc = cuda_ok(cudaMemcpyAsync(host_emitted, x->ws + x->L.emitted, c.B * W * 4, cudaMemcpyDeviceToHost, st));

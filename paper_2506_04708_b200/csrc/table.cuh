@@ -361,12 +361,8 @@ __device__ __forceinline__ void load_fresh(const UpdateParams& p, long long i, i
   }
 }
 
-__global__ void __launch_bounds__(APPLY_WARPS * 32) update_apply_kernel(const UpdateParams p) {
-  __shared__ SlotImage s_img[APPLY_WARPS];
-  const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
-  const long long g = (long long)blockIdx.x * APPLY_WARPS + warp;
-  pdl_trigger();
-  pdl_wait();  // records and slot marks come from stage 1
+// Record g (order-major index) by one warp; img is the warp's working image of the slot.
+__device__ __forceinline__ void apply_record(const UpdateParams& p, const long long g, SlotImage* img, const int lane) {
   if (g >= p.n_rows * p.n_max) return;
   // order-major, so that the warps of a block work on neighbouring rows of one order
   const int n = (int)(g / p.n_rows) + 1;
@@ -391,7 +387,6 @@ __global__ void __launch_bounds__(APPLY_WARPS * 32) update_apply_kernel(const Up
   const uint32_t word = line[lane];
   if (__shfl_sync(FULL, word, 6) != (uint32_t)row) return;  // another record leads this slot
   const uint32_t pending = __shfl_sync(FULL, word, 7);
-  SlotImage* img = &s_img[warp];
   if (lane == 4) img->count = word;
   if (lane == 5) img->n_items = word;
   if (lane >= 8 && lane < 8 + KMAX) img->ids[lane - 8] = (int)word;
@@ -439,6 +434,14 @@ __global__ void __launch_bounds__(APPLY_WARPS * 32) update_apply_kernel(const Up
     atomicAdd(&p.stats[ST_RECORDS], (unsigned long long)applied);
     if (fresh_slot) atomicAdd(&p.stats[ST_INSERTS], 1ull);
   }
+}
+
+__global__ void __launch_bounds__(APPLY_WARPS * 32) update_apply_kernel(const UpdateParams p) {
+  __shared__ SlotImage s_img[APPLY_WARPS];
+  const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+  pdl_trigger();
+  pdl_wait();  // records and slot marks come from stage 1
+  apply_record(p, (long long)blockIdx.x * APPLY_WARPS + warp, &s_img[warp], lane);
 }
 
 // ---------------------------------------------------------------------------

@@ -237,7 +237,8 @@ __device__ __forceinline__ double half_sum_d(double v) {
   return v;
 }
 
-__global__ void __launch_bounds__(K2_THREADS, 2) verify_kernel(const VerifyParams p) {
+// The verification of sequence b by one block of K2_THREADS threads.
+__device__ __forceinline__ void verify_block(const VerifyParams& p, const int b) {
   // per-node state, sized by the tree (verify_smem_bytes): target probabilities of the candidates, normaliser
   // reciprocals and offsets, the candidate lists, tree tokens and topology
   extern __shared__ __align__(16) unsigned char s_dyn[];
@@ -268,7 +269,6 @@ __global__ void __launch_bounds__(K2_THREADS, 2) verify_kernel(const VerifyParam
   __shared__ int s_ncand[TOPK_ROWS], s_nitems;
   __shared__ float s_floor[TOPK_ROWS];
 
-  const int b = blockIdx.x;
   const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
   const int N = p.N, K = p.K;
   const double cd = (double)p.c;
@@ -627,5 +627,7 @@ __global__ void __launch_bounds__(K2_THREADS, 2) verify_kernel(const VerifyParam
     }
   }
 }
+
+__global__ void __launch_bounds__(K2_THREADS, 2) verify_kernel(const VerifyParams p) { verify_block(p, (int)blockIdx.x); }
 
 }  // namespace stand
