@@ -252,6 +252,7 @@ __device__ __forceinline__ void verify_block(const VerifyParams& p, const int b)
   int* s_fc = s_cn + p.N;
   int* s_nch = s_fc + p.N;
   __shared__ int s_tail[ORDER_MAX];
+  __shared__ long long s_len;
   __shared__ double s_scan[K2_THREADS / 32];
   __shared__ int s_path[DEPTH_MAX + 1];
   __shared__ int s_emit[DEPTH_MAX + 1];
@@ -287,6 +288,7 @@ __device__ __forceinline__ void verify_block(const VerifyParams& p, const int b)
     s_cphi[(u) * KMAX + (t)] = p.cand_phi[(long long)b * N * K + i];
   }
   if (tid < p.n_max) s_tail[tid] = p.tail[b * p.n_max + tid];
+  if (tid == 32) s_len = p.len[b];  // read here so that the output phase does not wait for it
   __syncthreads();
 
   // ---- phase 1: the candidate logits are requested first (one round of gathers), the normalisers
@@ -308,17 +310,38 @@ __device__ __forceinline__ void verify_block(const VerifyParams& p, const int b)
       const int u = u0 + tid / ROW_LANES;
       const bool live = u < N;
       const float2* pairs = p.pairs + ((long long)b * N + (live ? u : 0)) * p.n_chunks;
+      // the pairs are read in batches of independent loads (a loop of load-then-use would pay one
+      // cache round trip per chunk)
+      constexpr int BATCH = 8;
       float mm = -INFINITY;
       if (live)
-        for (int ch = gl; ch < p.n_chunks; ch += ROW_LANES) mm = fmaxf(mm, pairs[ch].y);
+        for (int c0 = gl; c0 < p.n_chunks; c0 += BATCH * ROW_LANES) {
+          float y[BATCH];
+#pragma unroll
+          for (int k = 0; k < BATCH; ++k) {
+            const int ch = c0 + k * ROW_LANES;
+            y[k] = ch < p.n_chunks ? pairs[ch].y : -INFINITY;
+          }
+#pragma unroll
+          for (int k = 0; k < BATCH; ++k) mm = fmaxf(mm, y[k]);
+        }
 #pragma unroll
       for (int o = ROW_LANES / 2; o > 0; o >>= 1) mm = fmaxf(mm, __shfl_xor_sync(FULL, mm, o));
       const float om = chunk_offset(mm, p.c);  // the offset grows with the maximum
       double z0 = 0.0, z1 = 0.0;
       if (live)
-        for (int ch = gl; ch < p.n_chunks; ch += 2 * ROW_LANES) {
-          z0 += (double)chunk_mass_f(pairs[ch], p.c, om);
-          if (ch + ROW_LANES < p.n_chunks) z1 += (double)chunk_mass_f(pairs[ch + ROW_LANES], p.c, om);
+        for (int c0 = gl; c0 < p.n_chunks; c0 += BATCH * ROW_LANES) {
+          float2 v[BATCH];
+#pragma unroll
+          for (int k = 0; k < BATCH; ++k) {
+            const int ch = c0 + k * ROW_LANES;
+            v[k] = ch < p.n_chunks ? pairs[ch] : make_float2(0.0f, -INFINITY);  // an empty chunk has no mass
+          }
+#pragma unroll
+          for (int k = 0; k < BATCH; k += 2) {  // the same two running sums, in the same order, as one chunk at a time
+            z0 += (double)chunk_mass_f(v[k], p.c, om);
+            z1 += (double)chunk_mass_f(v[k + 1], p.c, om);
+          }
         }
       double z = z0 + z1;
 #pragma unroll
@@ -528,7 +551,7 @@ __device__ __forceinline__ void verify_block(const VerifyParams& p, const int b)
       win[p.n_max - 1] = s_emit[j];
     }
     for (int i = 0; i < p.n_max; ++i) p.tail[b * p.n_max + i] = win[i];
-    p.len[b] += m + 1;
+    p.len[b] = s_len + m + 1;
     p.n_path[b] = m + 1;
     if (p.n_emitted_user) p.n_emitted_user[b] = m + 1;
     atomicAdd(&p.stats[ST_EMITTED], (unsigned long long)(m + 1));
