@@ -392,6 +392,39 @@ def test_sharded_contexts_equal_the_unsharded_one(deterministic):
         sh.stand.close()
 
 
+@pytest.mark.parametrize("B", [1, 3])
+def test_host_buffer_step_equals_the_device_buffer_step(B):
+    """stand_step_host (logits in pinned host memory, results copied back, stream synchronised) against
+    stand_step on device buffers: same emitted tokens, trees and tables, step by step."""
+    torch = _torch()
+    from paper_2506_04708_b200.binding import Stand, StandError
+    w = inputs.scaled(inputs.WORKLOADS["cfg1"], B=B, steps=20, dtype=inputs.DTYPE_BF16)
+    parent = inputs.topology(w.N, w.D, w.kb)
+    depth = inputs.node_depths(parent)
+    streams = inputs.token_streams(w, 9, 300)
+    mk = lambda staging: Stand(w.B, w.N, w.V, w.topk, w.order_max, w.dtype, w.T, 9, 1 << 14, parent, host_staging=staging)
+    dev, host = mk(False), mk(True)
+    tail = torch.from_numpy(streams[:, 5:8].copy())
+    lens = np.full(w.B, 8, np.int64)
+    dev.reset_sequences(tail, torch.from_numpy(lens))
+    host.reset_sequences(tail, torch.from_numpy(lens))
+    h_em = torch.empty((w.B, dev.D + 1), dtype=torch.int32).pin_memory()
+    h_ne = torch.empty(w.B, dtype=torch.int32).pin_memory()
+    h_tr = torch.empty((w.B, w.N), dtype=torch.int32).pin_memory()
+    for s in range(20):
+        logits = inputs.logits_numpy(w, streams, lens, depth, s, 9, "p80")
+        h_logits = torch.from_numpy(logits.view(np.int16)).view(torch.bfloat16).pin_memory()
+        em, ne, tr = (t.cpu().numpy() for t in dev.step(harness.to_device_logits(logits)))
+        host.step_host(h_logits, h_em, h_ne, h_tr)
+        assert np.array_equal(em, h_em.numpy()) and np.array_equal(ne, h_ne.numpy()) and np.array_equal(tr, h_tr.numpy()), s
+        lens = dev.state_dump()["len"]
+    assert dev.table_dict() == host.table_dict()
+    # a context made without the staging buffer refuses the host entry point
+    with pytest.raises(StandError):
+        dev.step_host(h_logits, h_em, h_ne, h_tr)
+    dev.close(); host.close()
+
+
 def test_table_persists_across_trajectories_and_resume_from_a_checkpoint():
     """Sec. 5.1: the N-gram module is kept across trajectories (stand_reset_sequences restarts the sequences only).
     And a run resumed in a fresh context from dumped table + state continues exactly like the original."""
