@@ -277,13 +277,14 @@ def test_node_acceptance_counters_and_tree_optimisation():
         loop2.close()
 
 
-def test_full_initial_tree_to_eighty_nodes():
+@pytest.mark.parametrize("B", [3, 1])  # a batch, and the paper's own setting: one sequence (the two-launch step)
+def test_full_initial_tree_to_eighty_nodes(B):
     """The paper's procedure at its own sizes (Sec. 4.2, App. A.1): all 625 nodes of Algorithm 1's tree, acceptance
     counts over a run, the 80 most accepted nodes kept."""
     from paper_2506_04708_b200 import binding
     parent, depth, _, total = binding.initial_tree()
     assert total == 625 and len(parent) == 625
-    w = inputs.Workload("init625", 3, 625, int(depth.max()), 8, 2000, inputs.DTYPE_BF16, 0.6, 4, 10, 25, 1 << 14, 2.0, 0.7,
+    w = inputs.Workload("init625", B, 625, int(depth.max()), 8, 2000, inputs.DTYPE_BF16, 0.6, 4, 10, 25, 1 << 14, 2.0, 0.7,
                         24, 1.05)
     loop = harness.ClosedLoop(w, seed=4, peak_mode="p80", parent=parent)
     try:
@@ -296,7 +297,7 @@ def test_full_initial_tree_to_eighty_nodes():
     finally:
         loop.close()
     assert len(small) == 80 and small[0] == -1
-    w2 = inputs.Workload("opt80", 3, 80, int(inputs.node_depths(small).max()), 8, 2000, inputs.DTYPE_BF16, 0.6, 4, 10, 20,
+    w2 = inputs.Workload("opt80", B, 80, int(inputs.node_depths(small).max()), 8, 2000, inputs.DTYPE_BF16, 0.6, 4, 10, 20,
                          1 << 14, 2.0, 0.7, 24, 1.05)
     loop2 = harness.ClosedLoop(w2, seed=4, peak_mode="p80", parent=small)
     try:
