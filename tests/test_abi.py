@@ -97,6 +97,13 @@ def test_workspace_bytes_and_rejections(lib):
     assert lib.stand_init(None, C.c_void_p(0x1000), need, C.byref(h)) == -1
     assert lib.stand_destroy(None) == -1
     assert lib.stand_step(None, None, None, None, None, None) == -1
+    # sequence sharding: a negative first-sequence index, or one that overflows with B, is not a configuration
+    assert bad(seq_base=-1) == 0
+    assert bad(seq_base=2**31 - 1) == 0
+    assert bad(seq_base=12345) == need
+    assert lib.stand_export_records(None, None, None, None, None) == -1
+    assert lib.stand_skip_update(None) == -1
+    assert lib.stand_ngram_update_bulk(None, None, None, None, 0, None) == -1
 
 
 def test_strerror_and_scratch_size(lib):
