@@ -154,8 +154,9 @@ int stand_skip_update(stand_ctx* ctx);
  * NULL) and keeps the tree and the candidate lists for the next verification. */
 int stand_draft_tree(stand_ctx* ctx, int32_t* dev_tree_tokens, void* cu_stream);
 
-/* verify -> update -> draft on one stream, no host synchronisation: four kernel launches for a batch, two
- * for a single sequence (B = 1: the row pass, then verification, update and drafting in one block). */
+/* verify -> update -> draft on one stream, no host synchronisation: two kernel launches for up to 16
+ * sequences (the row pass, then verification, update and drafting in one block, or in one thread-block
+ * cluster with a block per sequence), four for larger batches. */
 int stand_step(stand_ctx* ctx, const void* dev_logits, int32_t* dev_emitted, int32_t* dev_n_emitted,
                int32_t* dev_tree_tokens, void* cu_stream);
 

@@ -112,6 +112,7 @@ struct stand_ctx {
   uint64_t launches;
   cudaStream_t last_stream;
   int max_probe;
+  int tail_form;  // 0: three kernels; 1: one block (single sequence); 2: one cluster of B blocks
   float c;  // log2(e) / T
   cudaEvent_t ev_before, ev_after;  // optional timing hook around the row pass
   cudaEvent_t ev_stage[5];          // optional timing hook at the stage boundaries of a step
@@ -163,6 +164,10 @@ int prepare_device(int* sm_count) {
       return STAND_E_CUDA;
     if (cudaFuncSetAttribute(tail_single_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)verify_smem_bytes(NODES_MAX)) !=
         cudaSuccess)
+      return STAND_E_CUDA;
+    if (cudaFuncSetAttribute(tail_cluster_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)verify_smem_bytes(NODES_MAX)) !=
+            cudaSuccess ||
+        cudaFuncSetAttribute(tail_cluster_kernel, cudaFuncAttributeNonPortableClusterSizeAllowed, 1) != cudaSuccess)
       return STAND_E_CUDA;
     g_sm_count[dev].store(sms, std::memory_order_relaxed);
     g_k1_ready[dev].store(1, std::memory_order_release);
@@ -219,6 +224,48 @@ int launch_dependent(void (*kernel)(P), unsigned grid, unsigned block, cudaStrea
   cfg.attrs = attr;
   cfg.numAttrs = 1;
   return cuda_ok(cudaLaunchKernelEx(&cfg, kernel, params));
+}
+
+// The same, as one thread-block cluster of `grid` blocks.
+template <typename P>
+int launch_dependent_cluster(void (*kernel)(P), unsigned grid, unsigned block, cudaStream_t st, const P& params, size_t smem) {
+  cudaLaunchConfig_t cfg = {};
+  cfg.gridDim = dim3(grid);
+  cfg.blockDim = dim3(block);
+  cfg.dynamicSmemBytes = smem;
+  cfg.stream = st;
+  cudaLaunchAttribute attr[2];
+  attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+  attr[0].val.programmaticStreamSerializationAllowed = 1;
+  attr[1].id = cudaLaunchAttributeClusterDimension;
+  attr[1].val.clusterDim.x = grid;
+  attr[1].val.clusterDim.y = 1;
+  attr[1].val.clusterDim.z = 1;
+  cfg.attrs = attr;
+  cfg.numAttrs = 2;
+  return cuda_ok(cudaLaunchKernelEx(&cfg, kernel, params));
+}
+
+// Can one cluster of B tail blocks run on this device?  (Asked once, at stand_init.)
+bool cluster_tail_fits(int B, size_t smem) {
+  if (B < 2 || B > TAIL_CLUSTER_MAX) return false;
+  cudaLaunchConfig_t cfg = {};
+  cfg.gridDim = dim3((unsigned)B);
+  cfg.blockDim = dim3(K2_THREADS);
+  cfg.dynamicSmemBytes = smem;
+  cudaLaunchAttribute attr[1];
+  attr[0].id = cudaLaunchAttributeClusterDimension;
+  attr[0].val.clusterDim.x = (unsigned)B;
+  attr[0].val.clusterDim.y = 1;
+  attr[0].val.clusterDim.z = 1;
+  cfg.attrs = attr;
+  cfg.numAttrs = 1;
+  int clusters = 0;
+  if (cudaOccupancyMaxActiveClusters(&clusters, tail_cluster_kernel, &cfg) != cudaSuccess) {
+    cudaGetLastError();  // not an error of the library: the batch takes the three-kernel form
+    return false;
+  }
+  return clusters >= 1;
 }
 
 UpdateParams update_params(stand_ctx* x, long long n_rows, const int* ctxw, const int* ids, const float* probs,
@@ -340,19 +387,20 @@ bool timing_hooks(const stand_ctx* x) {
   return false;
 }
 
-// One whole step on a stream.  A single sequence takes two launches (row pass, then its whole tail in one
-// block); batches take four.
+// One whole step on a stream.  A single sequence and a small batch take two launches (row pass, then the
+// whole tail in one block or one cluster); larger batches take four.
 int run_step(stand_ctx* x, const void* logits, int32_t* emitted, int32_t* n_emitted, int32_t* tree_user, cudaStream_t st) {
   const stand_config& c = x->cfg;
-  if (c.B == 1 && !timing_hooks(x)) {
-    int rc = launch_row_pass(logits, (long long)c.N, c.V, c.dtype, x->d.n_chunks, x->c, x->at<float2>(x->L.pairs),
+  if (x->tail_form != 0 && !timing_hooks(x)) {
+    int rc = launch_row_pass(logits, (long long)c.B * c.N, c.V, c.dtype, x->d.n_chunks, x->c, x->at<float2>(x->L.pairs),
                              x->at<int>(x->L.status), st, true);
     if (rc) return rc;
     x->step += 1;
     TailParams t;
     t.v = verify_params(x, logits, emitted, n_emitted, true);
     t.d = draft_params(x, tree_user);
-    rc = launch_dependent(tail_single_kernel, 1u, K2_THREADS, st, t, verify_smem_bytes(c.N));
+    if (x->tail_form == 1) rc = launch_dependent(tail_single_kernel, 1u, K2_THREADS, st, t, verify_smem_bytes(c.N));
+    else rc = launch_dependent_cluster(tail_cluster_kernel, (unsigned)c.B, K2_THREADS, st, t, verify_smem_bytes(c.N));
     if (rc) return rc;
     x->launches += 2;
     x->pending = false;
@@ -430,6 +478,7 @@ int stand_init(const stand_config* cfg, void* dev_workspace, size_t bytes, stand
   x->launches = 0;
   x->last_stream = 0;
   x->max_probe = cfg->max_probe > 0 ? cfg->max_probe : 96;
+  x->tail_form = cfg->B == 1 ? 1 : (cluster_tail_fits(cfg->B, verify_smem_bytes(cfg->N)) ? 2 : 0);
   x->ev_before = nullptr;
   x->ev_after = nullptr;
   for (int i = 0; i < 5; ++i) x->ev_stage[i] = nullptr;

@@ -1,4 +1,5 @@
-// Single-sequence step tail: verification, table update and drafting in one thread block.
+// Step tail without kernel boundaries: verification, table update and drafting in one thread block (a single
+// sequence) or one thread-block cluster (a small batch).
 #pragma once
 #include "common.cuh"
 #include "draft.cuh"
@@ -7,28 +8,46 @@
 
 namespace stand {
 
-// A whole step's tail for ONE sequence in one block: verification (with stage 1 of the update), stage 2 of
-// the update, drafting.  With a single sequence every ordering the three kernels get from their launch
-// boundaries is a block barrier here, which saves two kernel boundaries on the latency path.
+// A whole step's tail without kernel boundaries, for a single sequence (one block) or a small batch (one
+// block per sequence, all blocks in ONE thread-block cluster): verification with stage 1 of the update,
+// stage 2 of the update, drafting.  Where the batch form relies on a kernel boundary ("every sequence has
+// located its records", "the table is up to date") this form has a block barrier, or the hardware barrier
+// of the cluster, whose release/acquire pair also orders the blocks' global-memory writes.
 static_assert(K2_THREADS == K4_THREADS && K2_THREADS == APPLY_WARPS * 32, "one block shape for the three stages");
+constexpr int TAIL_CLUSTER_MAX = 16;  // largest cluster the hardware offers (beyond 8 it has to be asked for)
 struct TailParams {
   VerifyParams v;  // fuse_locate set; v.upd describes this step's records
   DraftParams d;
 };
-__global__ void __launch_bounds__(K2_THREADS) tail_single_kernel(const TailParams p) {
+
+template <bool CLUSTER>
+__device__ __forceinline__ void tail_barrier() {
+  if (CLUSTER) asm volatile("barrier.cluster.arrive.release.aligned;\n\tbarrier.cluster.wait.acquire.aligned;" ::: "memory");
+  else __syncthreads();
+}
+
+template <bool CLUSTER>
+__device__ __forceinline__ void tail_body(const TailParams& p, const int b) {
   __shared__ SlotImage s_img[APPLY_WARPS];
-  verify_block(p.v, 0);
-  __syncthreads();  // records, slot marks and the advanced tail are visible to the whole block
+  verify_block(p.v, b);
+  tail_barrier<CLUSTER>();  // records, slot marks and the advanced tails of all sequences are visible
   const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
-  // only the rows of the accepted path carry records: (row, order) pairs of the first n_path rows
-  const int live_rows = p.v.n_path[0];
+  // this block applies the records of its own sequence; only the rows of the accepted path carry any:
+  // (row, order) pairs of the first n_path rows.  (A slot's records are applied by the warp that holds its
+  // lowest row, whichever block that is: the canonical order does not depend on who runs what.)
+  const int W1 = p.v.D + 1;
+  const int live_rows = p.v.n_path[b];
   const int n_rec = live_rows * p.v.upd.n_max;
   for (int r = warp; r < n_rec; r += APPLY_WARPS) {
     const int n = r / live_rows, row = r - n * live_rows;
-    apply_record(p.v.upd, (long long)n * p.v.upd.n_rows + row, &s_img[warp], lane);
+    apply_record(p.v.upd, (long long)n * p.v.upd.n_rows + (long long)b * W1 + row, &s_img[warp], lane);
   }
-  __syncthreads();  // the table is up to date
-  draft_block<false>(p.d, 0);
+  tail_barrier<CLUSTER>();  // the table is up to date
+  draft_block<false>(p.d, b);
 }
+
+__global__ void __launch_bounds__(K2_THREADS) tail_single_kernel(const TailParams p) { tail_body<false>(p, 0); }
+// Launched as one cluster of B blocks (cluster dimension = grid dimension = B <= TAIL_CLUSTER_MAX).
+__global__ void __launch_bounds__(K2_THREADS) tail_cluster_kernel(const TailParams p) { tail_body<true>(p, (int)blockIdx.x); }
 
 }  // namespace stand
