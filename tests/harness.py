@@ -122,9 +122,17 @@ class ClosedLoop:
             if ne_g[b] != ne_o[b] or not np.array_equal(em_g[b], em_o[b]) or not np.array_equal(tr_g[b], tr_o[b]):
                 bad_b.add(b)
         if bad_b:
+            # A sequence may differ from the oracle only if one of its own decisions (accept test, final sample,
+            # Gumbel selection) was logged with a margin below the tolerance, or if the two tables differ at a
+            # context whose truncation was decided by less than the tolerance (its drafts then read other candidates).
+            table_diffs = None
             for b in sorted(bad_b):
-                excuse = low[(low[:, 1] == b) | (low[:, 0] == so.MARGIN_MERGE)]
-                if len(excuse) == 0:
+                excused = len(low[low[:, 1] == b]) > 0
+                if not excused and self.low_margin_keys:
+                    if table_diffs is None:
+                        table_diffs = compare_tables(self.gpu.table_dict(), self.orc.table(), value_tol(w.dtype))
+                    excused = any(d[0] == "ids" and d[1] in self.low_margin_keys for d in table_diffs)
+                if not excused:
                     self.hard.append((self.step_no, b, em_g[b].tolist(), em_o[b].tolist(), tr_g[b].tolist(),
                                       tr_o[b].tolist()))
                 else:
