@@ -330,6 +330,7 @@ void merge_entry(Entry& e, const std::vector<std::pair<int, double>>& fresh, int
 struct Oracle {
   int B, N, V, K, n_max, dtype;
   int deterministic = 0;  // 1: deterministic drafting (Sec. 3.2), 0: stochastic (Sec. 4.2)
+  int seq_base = 0;       // global index of sequence 0: the random-number counters use seq_base + b
   double T;
   uint64_t seed;
   std::vector<int> parent, depth;
@@ -378,7 +379,7 @@ struct Oracle {
       std::vector<int> drafted_nodes, drafted_tokens;
       for (int c : children[u])
         if (tree[b][c] >= 0) { drafted_nodes.push_back(c); drafted_tokens.push_back(tree[b][c]); }
-      const double u_final = uniform_half_open(random_u24(seed, b, step, u, SLOT_FINAL));
+      const double u_final = uniform_half_open(random_u24(seed, (uint32_t)(seq_base + b), step, u, SLOT_FINAL));
       MarginRec mr;
       mr.b = b; mr.node = u; for (int i = 0; i < 4; ++i) mr.key[i] = -1;
       if (drafted_nodes.empty()) {
@@ -390,7 +391,7 @@ struct Oracle {
       }
       std::vector<double> u_acc(drafted_nodes.size());
       for (size_t j = 0; j < drafted_nodes.size(); ++j)
-        u_acc[j] = uniform_half_open(random_u24(seed, b, step, u, (uint32_t)j));
+        u_acc[j] = uniform_half_open(random_u24(seed, (uint32_t)(seq_base + b), step, u, (uint32_t)j));
       int resampled = -1;
       std::vector<double> am;
       double fm = 1.0;
@@ -491,7 +492,7 @@ struct Oracle {
         if (it.second > 0.0) {
           ids.push_back(it.first);
           phis.push_back(it.second);
-          U.push_back(uniform_open(random_u24(seed, b, step, u, SLOT_GUMBEL | (uint32_t)it.first)));
+          U.push_back(uniform_open(random_u24(seed, (uint32_t)(seq_base + b), step, u, SLOT_GUMBEL | (uint32_t)it.first)));
         }
       double mg;
       std::vector<int> chosen = deterministic ? most_probable(ids, phis, m, &mg) : gumbel_top(ids, phis, U, m, &mg);
@@ -605,6 +606,8 @@ void* so_create(int B, int N, int V, int topk, int order_max, int dtype, double 
   return o;
 }
 void so_set_deterministic(void* h, int on) { ((Oracle*)h)->deterministic = on ? 1 : 0; }
+// A batch split over several contexts: this context's sequence b is sequence seq_base + b of the batch.
+void so_set_seq_base(void* h, int base) { ((Oracle*)h)->seq_base = base; }
 void so_destroy(void* h) { delete (Oracle*)h; }
 int so_depth(void* h) { return ((Oracle*)h)->D; }
 

@@ -116,7 +116,7 @@ MARGIN_ACCEPT, MARGIN_FINAL, MARGIN_GUMBEL, MARGIN_MERGE = 0, 1, 2, 3
 
 
 class Oracle:
-    def __init__(self, B, N, V, topk, order_max, dtype, temperature, seed, parent, deterministic=False):
+    def __init__(self, B, N, V, topk, order_max, dtype, temperature, seed, parent, deterministic=False, seq_base=0):
         self.B, self.N, self.V, self.K, self.n_max, self.dtype = B, N, V, topk, order_max, dtype
         self.parent = np.ascontiguousarray(parent, np.int32)
         assert len(self.parent) == N
@@ -127,6 +127,8 @@ class Oracle:
         self.D = lib().so_depth(self.h)
         if deterministic:
             lib().so_set_deterministic(self.h, 1)
+        if seq_base:
+            lib().so_set_seq_base(self.h, int(seq_base))
 
     def close(self):
         if self.h:

@@ -68,7 +68,7 @@ class ClosedLoop:
     """Runs the same seeded workload through both sides, step by step."""
 
     def __init__(self, w, seed=0, peak_mode="add8", table_slots=None, prompt=8, device="cuda:0", device_logits=False,
-                 parent=None, deterministic=False, **stand_kw):
+                 parent=None, deterministic=False, seq_base=0, **stand_kw):
         from paper_2506_04708_b200.binding import Stand
         self.w, self.seed, self.peak_mode = w, seed, peak_mode
         self.parent = inputs.topology(w.N, w.D, w.kb) if parent is None else np.ascontiguousarray(parent, np.int32)
@@ -76,9 +76,9 @@ class ClosedLoop:
         self.streams = inputs.token_streams(w, seed, prompt + (w.steps + 2) * (w.D + 2))
         slots = table_slots or w.table_slots
         self.gpu = Stand(w.B, w.N, w.V, w.topk, w.order_max, w.dtype, w.T, seed, slots, self.parent, device=device,
-                         deterministic=deterministic, **stand_kw)
+                         deterministic=deterministic, seq_base=seq_base, **stand_kw)
         self.orc = so.Oracle(w.B, w.N, w.V, w.topk, w.order_max, w.dtype, w.T, seed, self.parent,
-                             deterministic=deterministic)
+                             deterministic=deterministic, seq_base=seq_base)
         import torch
         tail = np.full((w.B, w.order_max), -1, np.int32)
         take = min(prompt, w.order_max)

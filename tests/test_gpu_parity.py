@@ -345,6 +345,25 @@ def test_stage_calls_equal_the_fused_step(B):
     a.close(); b.close()
 
 
+def test_sequence_base_against_the_oracle():
+    """A context whose sequences are numbers 5.. of a larger batch (seq_base = 5): its random numbers are those
+    of sequences 5.., on both sides; and they are not those of sequences 0..."""
+    w = inputs.Workload("tiny", 3, 16, 4, 3, 1000, inputs.DTYPE_BF16, 0.9, 3, 6, 60, 1 << 12, 2.0, 0.7, 12, 1.1)
+    emitted = {}
+    for base in (5, 0):
+        loop = harness.ClosedLoop(w, seed=2, peak_mode="p80", seq_base=base)
+        try:
+            seen = []
+            for _ in range(w.steps):
+                seen.append(loop.step()[0].copy())
+            assert loop.hard == [] and loop.check_state_and_table() == []
+            assert loop.tolerated <= 2
+            emitted[base] = np.stack(seen)
+        finally:
+            loop.close()
+    assert not np.array_equal(emitted[5], emitted[0])
+
+
 @pytest.mark.parametrize("deterministic", [False, True])
 def test_sharded_contexts_equal_the_unsharded_one(deterministic):
     """A batch of 6 sequences split 2 + 4 over two contexts (seq_base 0 and 2), each with its own copy of the

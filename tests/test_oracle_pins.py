@@ -485,3 +485,29 @@ def test_update_feeds_only_the_accepted_path_in_order():
     st = o.state()
     assert list(st["tail"][0]) == [5, em[0, 0]] and st["len"][0] == 3 and tree[0, 0] == em[0, 0]
     o.close()
+
+
+def test_sequence_base_offsets_the_counter_of_every_draw():
+    """A context that holds sequences seq_base.. of a larger batch draws the random numbers of those sequences
+    (counter word 0 = seq_base + b): with a one-node tree every step is one inverse-CDF draw, recomputed here
+    from the published uniform of sequence seq_base + b."""
+    V, T, seed, base = 64, 0.8, 11, 3
+    rng = np.random.default_rng(5)
+    parent = np.array([-1], np.int32)
+    o = so.Oracle(2, 1, V, 4, 2, 0, T, seed, parent, seq_base=base)
+    o.reset_sequences(np.full((2, 2), 1, np.int32), np.full(2, 4, np.int64))
+    shifted = 0
+    for step in range(1, 21):
+        logits = rng.normal(0, 2, size=(2, 1, V)).astype(np.float32)
+        em, ne, _ = o.step(logits)
+        assert list(ne) == [1, 1]
+        for b in range(2):
+            z = logits[b, 0].astype(np.float64) / np.float64(np.float32(T))
+            p = np.exp(z - z.max())
+            cdf = np.cumsum(p)
+            pick = lambda seq: int(np.searchsorted(cdf, so.uniform(seed, seq, step, 0, 0x40000000) * cdf[-1], side="right"))
+            assert em[b, 0] == pick(base + b)
+            shifted += em[b, 0] != pick(b)
+    assert shifted > 20  # and not those of sequences 0, 1
+    o.take_margins()
+    o.close()
