@@ -41,6 +41,9 @@ def main():
     try:
         for s in range(steps):
             loop.step()
+            if (s + 1) % max(1, steps // 16) == 0:  # progress, so that a run cut short still says how far it got
+                print(json.dumps({"progress": s + 1, "hard_mismatches": len(loop.hard), "tolerated_low_margin": loop.tolerated,
+                                  "seconds": round(time.time() - t0, 1)}), file=sys.stderr, flush=True)
             if args.check_every and (s + 1) % args.check_every == 0 and s + 1 < steps:
                 checks.append(len(loop.check_state_and_table()))
         final = loop.check_state_and_table()
