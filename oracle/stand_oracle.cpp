@@ -28,10 +28,12 @@
 // Pins (tests marked "not gpu"): Philox known-answer vectors; softmax and
 // top-k against library routines; losslessness of verification by black-box
 // threshold search and by chi-square; Gumbel-Top-K against the Plackett-Luce
-// closed form; table contents against a recount of the token stream; hand
-// cases for the merge and the lookup order.  Parity unpinned: the canonical
-// order of same-step updates from different sequences (a convention, the
-// paper fixes none).
+// closed form; table contents against a recount of the token stream, both
+// for bulk rows and for whole steps on one-hot targets (which pins the
+// pairing of accepted-path rows with their context windows); hand cases for
+// the merge, the lookup order and the contexts of nodes deep in the tree.
+// Parity unpinned: the canonical order of same-step updates from different
+// sequences (a convention, the paper fixes none).
 //
 // Everything floating point is double.  Nothing is blocked, fused or
 // reordered: vectors over the whole vocabulary are used wherever the

@@ -511,3 +511,110 @@ def test_sequence_base_offsets_the_counter_of_every_draw():
     assert shifted > 20  # and not those of sequences 0, 1
     o.take_margins()
     o.close()
+
+
+# ------------------------------- the update's pairing of rows and context windows (Sec. 4.1, Fig. "Overview")
+def _one_hot_logits(parent, streams, lens, V):
+    """Row (b, u) puts all its mass on the token that the stream holds at the position the row predicts
+    (len_b + depth(u)): exp(-1000) is zero in double precision, so every row is a one-hot distribution."""
+    depth = np.zeros(len(parent), int)
+    for u in range(1, len(parent)):
+        depth[u] = depth[parent[u]] + 1
+    x = np.zeros((len(streams), len(parent), V), np.float32)
+    for b in range(len(streams)):
+        for u in range(len(parent)):
+            x[b, u, streams[b][lens[b] + depth[u]]] = 1000.0
+    return x
+
+
+@pytest.mark.parametrize("B", [1, 3])
+def test_closed_loop_table_equals_a_recount_of_the_emitted_stream(B):
+    """Whole steps (verify -> update -> draft) on one-hot target rows: whatever is drafted, the emitted tokens are
+    the stream's, accepted paths are several nodes long once contexts repeat, and the table must hold, under every
+    order, exactly the follower frequencies of the emitted text (Sec. 4.1: "when the language model generates
+    'I am Bob' we store the distribution" of the token after it).  The recount below knows nothing about trees or
+    paths: it pins which row is paired with which context window along an accepted path."""
+    rng = np.random.default_rng(40 + B)
+    V, K, n_max = 40, 6, 3
+    parent = np.array([-1, 0, 0, 1, 1, 2, 3, 3, 6, 8], np.int32)  # branching: a node's index is not its depth
+    prompt, total = 5, 700
+    # text made of a few recurring phrases over five tokens: inside a phrase a context has one follower and the
+    # drafts run deep, at a phrase boundary it has several and drafts are rejected
+    phrases = [list(3 + 7 * rng.integers(0, 5, rng.integers(5, 10))) for _ in range(5)]
+    streams = []
+    for _ in range(B):
+        text = []
+        while len(text) < total:
+            text += phrases[rng.integers(0, len(phrases))]
+        streams.append(text)
+    o = so.Oracle(B, len(parent), V, K, n_max, 0, 1.0, 17, parent)
+    tail = np.array([s[prompt - n_max:prompt] for s in streams], np.int32)
+    lens = np.full(B, prompt, np.int64)
+    o.reset_sequences(tail, lens)
+    deep = 0
+    for _ in range(120):
+        em, ne, _ = o.step(_one_hot_logits(parent, streams, lens, V))
+        for b in range(B):
+            assert list(em[b, :ne[b]]) == streams[b][lens[b]:lens[b] + ne[b]]  # lossless on one-hot targets
+        deep += int((ne >= 3).sum())
+        lens = lens + ne
+    o.take_margins()
+    assert deep > 20 * B  # accepted paths with j >= 2 are the rule, not the exception
+    assert np.array_equal(o.state()["len"], lens)
+    want = {}
+    for b in range(B):
+        for t in range(prompt, int(lens[b])):
+            for n in range(1, n_max + 1):
+                key = tuple(int(v) for v in streams[b][t - n:t])
+                want.setdefault(key, {}).setdefault(int(streams[b][t]), 0)
+                want[key][int(streams[b][t])] += 1
+    got = o.table()
+    assert set(got) == set(want)
+    for key, followers in want.items():
+        cnt, items = got[key]
+        n_seen = sum(followers.values())
+        assert cnt == n_seen
+        positive = {t: v for t, v in items.items() if v > 0}
+        assert set(positive) == set(followers)
+        for t, c in followers.items():
+            assert abs(positive[t] - c / n_seen) < 1e-12
+    o.close()
+
+
+def test_deep_nodes_are_drafted_from_the_tail_plus_the_tokens_on_their_own_path():
+    """Sec. 4.2, "for each position in the draft tree": the context of a node below depth 1 is the sequence
+    followed by the tokens drafted on the way from the root to that node.  Here every lookup that matters can only
+    hit through such a context, and the two branches of the tree must each continue their own token."""
+    parent = np.array([-1, 0, 0, 1, 2, 3, 4], np.int32)  # two children of the root, each heads a chain of three
+    V, K, n_max = 100, 4, 2
+
+    def feed(o, window, ids, times=1):
+        i = np.full((1, K), -1, np.int32)
+        p = np.zeros((1, K), np.float32)
+        i[0, :len(ids)] = ids
+        p[0, :len(ids)] = 1.0 / len(ids)
+        for _ in range(times):
+            o.update_bulk(np.array([window], np.int32), i, p)
+
+    orders_seen = set()
+    for seed in range(8):
+        o = so.Oracle(1, len(parent), V, K, n_max, 0, 1.0, seed, parent)
+        feed(o, [6, 7], [20, 21])        # after (6, 7): 20 or 21
+        feed(o, [7, 20], [50])           # after (7, 20): 50      after (7, 21): 51
+        feed(o, [7, 21], [51])
+        feed(o, [20, 50], [60])          # after (20, 50): 60     after (21, 51): 61
+        feed(o, [21, 51], [61])
+        # the shorter contexts alone point elsewhere: a lookup that loses the path's earlier token is led astray
+        for tok, wrong in ((20, 40), (21, 41), (50, 42), (51, 43)):
+            feed(o, [9, tok], [wrong], times=5)
+        o.reset_sequences(np.array([[6, 7]], np.int32), np.array([2]))
+        tree = o.draft()[0]
+        assert tree[0] == 7 and sorted(tree[1:3]) == [20, 21]
+        orders_seen.add(tuple(tree[1:3]))
+        for head, mid, leaf in ((1, 3, 5), (2, 4, 6)):
+            assert tree[mid] == {20: 50, 21: 51}[tree[head]]   # context (7, tree[head]): tail + one path token
+            assert tree[leaf] == {50: 60, 51: 61}[tree[mid]]   # context (tree[head], tree[mid]): path tokens only
+        st = o.state()
+        assert st["cand_n"][0, 1] == 1 and st["cand_id"][0, 1, 0] == tree[3]  # the snapshot is the bigram's list
+        o.close()
+    assert len(orders_seen) == 2  # both Gumbel orders of the root's children occurred
