@@ -95,26 +95,18 @@ def test_maximum_sizes():
 
 
 def test_constant_logits_through_the_whole_step():
-    """Every row constant: the uniform target distribution, all top-k ties broken by id, through verify, update, draft."""
-    torch = _torch()
-    from paper_2506_04708_b200.binding import Stand
-    w = inputs.scaled(inputs.WORKLOADS["cfg1"], B=2, V=3000)
-    parent = inputs.topology(w.N, w.D, w.kb)
-    gpu = Stand(w.B, w.N, w.V, w.topk, w.order_max, w.dtype, w.T, 3, 1 << 12, parent)
-    orc = so.Oracle(w.B, w.N, w.V, w.topk, w.order_max, w.dtype, w.T, 3, parent)
-    tail = np.array([[1, 2, 3], [4, 5, 6]], np.int32)
-    lens = np.full(w.B, 8, np.int64)
-    gpu.reset_sequences(torch.from_numpy(tail), torch.from_numpy(lens))
-    orc.reset_sequences(tail, lens)
+    """Every row constant: the uniform target distribution, all top-k ties broken by id, through verify, update,
+    draft; every sequence of every step is judged by the margin rule."""
+    w = inputs.scaled(inputs.WORKLOADS["cfg1"], B=2, V=3000, steps=6)
+    loop = harness.ClosedLoop(w, seed=3, table_slots=1 << 12, tail=np.array([[1, 2, 3], [4, 5, 6]], np.int32))
     logits = np.full((w.B, w.N, w.V), 0.5, np.float32)
-    for s in range(4):
-        em, ne, tr = (t.cpu().numpy() for t in gpu.step(harness.to_device_logits(logits)))
-        em_o, ne_o, tr_o = orc.step(logits)
-        _, margins = orc.take_margins()
-        if margins.size == 0 or margins.min() >= harness.MARGIN_TOL:
-            assert np.array_equal(em, em_o) and np.array_equal(ne, ne_o) and np.array_equal(tr, tr_o), s
-    assert harness.compare_tables(gpu.table_dict(), orc.table(), 1e-5) == []
-    gpu.close(); orc.close()
+    try:
+        for s in range(w.steps):
+            loop.step(logits)
+        assert loop.hard == [] and loop.tolerated <= 1
+        assert loop.check_state_and_table() == []
+    finally:
+        loop.close()
 
 
 # ------------------------------------------------------------- whole step, closed loop
