@@ -231,7 +231,10 @@ int stand_table_load(stand_ctx* ctx, const int32_t* dev_keys, const uint32_t* de
 
 /* Sequence state export/import (checkpoint/resume): tails [B, order_max], lengths
  * [B] int64, tree tokens [B, N], candidate lists cand_n [B, N], cand_id / cand_phi
- * [B, N, topk], and the step counter (host).  load discards a pending verification. */
+ * [B, N, topk], and the step counter (host).  load discards a pending verification and checks the tree
+ * against the candidate lists: a drafted node whose token is outside the vocabulary, missing from its parent's
+ * candidate list (the draft distribution its verification divides by) or below an undrafted parent is cleared
+ * (-1) and counted in stand_stats.bad_tokens; candidate counts are clamped to [0, topk]. */
 int stand_state_dump(stand_ctx* ctx, int32_t* dev_tail, int64_t* dev_len, int32_t* dev_tree, int32_t* dev_cand_n,
                      int32_t* dev_cand_id, float* dev_cand_phi, uint32_t* host_step, void* cu_stream);
 int stand_state_load(stand_ctx* ctx, const int32_t* dev_tail, const int64_t* dev_len, const int32_t* dev_tree,
@@ -271,6 +274,15 @@ int stand_initial_tree(int32_t levels, int32_t* host_parent, int32_t* host_depth
  * stream by every later step at: before the row pass, after it, after the verification walk, after the
  * table update, after drafting.  A NULL array switches the hook off. */
 int stand_profile_stages(stand_ctx* ctx, void* const* events);
+
+/* Failure handling of the streaming kernel, made testable.  Every wait inside the kernels is bounded; when one
+ * runs out the kernel records it, lets its copies in flight land and returns, and the host sees
+ * stand_stats.wait_timeouts (or NaN / -1 results from stand_row_stats): the GPU context stays usable.  This
+ * call sets, for the whole process, how many polls the kernel's loader spends waiting for a free stage of its
+ * shared-memory ring: 1 .. 2^22 (the default, about a second); 0 makes its very first wait give up before
+ * anything was copied, which is how the tests reach the failure path; a negative value restores the default.
+ * Larger values are clamped: a wait cannot be made unbounded. */
+int stand_set_wait_limit(int64_t polls);
 
 /* How many kernels the library has launched through this context so far. */
 uint64_t stand_launch_count(const stand_ctx* ctx);

@@ -21,7 +21,7 @@ EXPORTS = [
     "stand_row_stats_scratch_bytes", "stand_row_stats", "stand_row_stats_static", "stand_get_stats",
     "stand_last_path", "stand_tree_depth", "stand_table_dump", "stand_table_load", "stand_state_dump",
     "stand_state_load", "stand_profile_row_pass", "stand_profile_stages", "stand_node_accepts", "stand_prune_tree",
-    "stand_initial_tree", "stand_launch_count", "stand_strerror",
+    "stand_initial_tree", "stand_launch_count", "stand_set_wait_limit", "stand_strerror",
 ]
 
 
@@ -99,6 +99,8 @@ def lib():
     L.stand_initial_tree.restype = C.c_int
     L.stand_launch_count.argtypes = [vp]
     L.stand_launch_count.restype = u64
+    L.stand_set_wait_limit.argtypes = [i64]
+    L.stand_set_wait_limit.restype = C.c_int
     L.stand_strerror.argtypes = [C.c_int]
     L.stand_strerror.restype = C.c_char_p
     for name in ["stand_init", "stand_destroy", "stand_reset_sequences", "stand_verify_tree", "stand_ngram_update",
@@ -234,11 +236,13 @@ class Stand:
         _check(lib().stand_draft_tree(self.h, _ptr(self.tree), _stream(stream)), "stand_draft_tree")
         return self.tree
 
-    def step(self, logits, stream=None):
+    def step(self, logits, stream=None, out=None):
+        """out: (emitted [B, D+1], n_emitted [B], tree [B, N]) int32 device tensors to write instead of the
+        context's own result tensors."""
         self._logits_ok(logits)
-        _check(lib().stand_step(self.h, _ptr(logits), _ptr(self.emitted), _ptr(self.n_emitted), _ptr(self.tree),
-                                _stream(stream)), "stand_step")
-        return self.emitted, self.n_emitted, self.tree
+        em, ne, tr = out if out is not None else (self.emitted, self.n_emitted, self.tree)
+        _check(lib().stand_step(self.h, _ptr(logits), _ptr(em), _ptr(ne), _ptr(tr), _stream(stream)), "stand_step")
+        return em, ne, tr
 
     def step_host(self, host_logits, host_emitted, host_n_emitted, host_tree, stream=None):
         """Host tensors in, host tensors out (pinned memory recommended); synchronises."""
@@ -408,6 +412,11 @@ def row_stats_static(logits, temperature, topk, out=None, stream=None):
                                             _ptr(vals), _ptr(probs), _stream(stream)), "stand_row_stats_static")
     (torch.cuda.current_stream() if stream is None else stream).synchronize()
     return out
+
+
+def set_wait_limit(polls):
+    """Polls the streaming kernel's loader spends on one wait (0: give up at once; negative: the default)."""
+    _check(lib().stand_set_wait_limit(int(polls)), "stand_set_wait_limit")
 
 
 def initial_tree(levels=20, capacity=None):

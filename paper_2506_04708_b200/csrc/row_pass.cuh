@@ -48,6 +48,7 @@ struct RowPassParams {
   float c;          // log2(e) / T
   float2* pairs;    // [rows, n_chunks]  (sum, chunk max)
   int* status;      // device word, set non-zero if a bounded wait ran out (may be null)
+  unsigned empty_wait_limit;  // polls the producer spends on one free-stage wait (SPIN_LIMIT unless a test lowers it)
 };
 
 __device__ __forceinline__ float ex2_approx(float x) {
@@ -195,8 +196,9 @@ __device__ __forceinline__ bool mbar_try_wait(uint32_t bar, uint32_t parity) {
   return ok != 0;
 }
 // Bounded wait; false if the limit ran out or another thread of the CTA already gave up.
-__device__ __forceinline__ bool mbar_wait_bounded(uint32_t bar, uint32_t parity, const volatile int* abort_flag) {
-  for (unsigned spin = 0; spin < SPIN_LIMIT; ++spin) {
+__device__ __forceinline__ bool mbar_wait_bounded(uint32_t bar, uint32_t parity, const volatile int* abort_flag,
+                                                  unsigned limit = SPIN_LIMIT) {
+  for (unsigned spin = 0; spin < limit; ++spin) {
     if (mbar_try_wait(bar, parity)) return true;
     if (*abort_flag) return false;
   }
@@ -245,7 +247,6 @@ __global__ void __launch_bounds__((CW + 1) * 32, CTAS) row_pass_kernel(const Row
   __shared__ volatile int s_abort;
 
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-  pdl_trigger();  // a dependent kernel may be scheduled as soon as resources free up; it waits for this grid's end
   const long long t0 = (long long)blockIdx.x * p.total_tiles / gridDim.x;
   const long long t1 = (long long)(blockIdx.x + 1) * p.total_tiles / gridDim.x;
   const int n_tiles = (int)(t1 - t0);
@@ -259,6 +260,10 @@ __global__ void __launch_bounds__((CW + 1) * 32, CTAS) row_pass_kernel(const Row
   }
   __syncthreads();
   pdl_wait();  // chained after the previous step: nothing is read or written before that step has ended
+  // Only now may the next kernel of this step be scheduled.  It reads sequence state (trees, candidate lists,
+  // tails) before its own wait, and its wait covers this grid only, not the step before: released earlier, it
+  // could run while the previous step's last kernel is still writing that state.
+  pdl_trigger();
   const size_t row_bytes = (size_t)p.V * TR::ESIZE;
   // tile coordinates advance without divisions
   long long row = t0 / p.tiles_per_row;
@@ -272,7 +277,7 @@ __global__ void __launch_bounds__((CW + 1) * 32, CTAS) row_pass_kernel(const Row
       uint32_t parity = 1;  // waiting for the phase before the first one succeeds at once
       const char* src_row = (const char*)p.logits + (size_t)row * row_bytes;
       for (int i = 0; i < n_tiles; ++i) {
-        if (!mbar_wait_bounded(smem_addr(&s_empty[s]), parity, &s_abort)) {
+        if (!mbar_wait_bounded(smem_addr(&s_empty[s]), parity, &s_abort, p.empty_wait_limit)) {
           if (!s_abort && p.status) atomicExch(p.status, K1_ERR_EMPTY_WAIT);
           s_abort = 1;
           break;

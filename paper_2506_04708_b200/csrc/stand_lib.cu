@@ -142,6 +142,7 @@ int launch_dependent(void (*kernel)(P), unsigned grid, unsigned block, cudaStrea
 
 // The streaming kernel needs more dynamic shared memory than the default limit: raise it once per device.
 constexpr int MAX_DEVICES = 64;
+std::atomic<unsigned> g_empty_wait_limit{SPIN_LIMIT};  // stand_set_wait_limit
 std::atomic<int> g_k1_ready[MAX_DEVICES];
 std::atomic<int> g_sm_count[MAX_DEVICES];
 
@@ -180,6 +181,7 @@ int launch_row_pass(const void* logits, long long rows, int V, int dtype, int n_
                     cudaStream_t st, bool chain = false) {
   RowPassParams rp;
   rp.logits = logits; rp.rows = rows; rp.V = V; rp.n_chunks = n_chunks; rp.c = c; rp.pairs = pairs; rp.status = status;
+  rp.empty_wait_limit = g_empty_wait_limit.load(std::memory_order_relaxed);
   const int tile_chunks = dtype == STAND_DTYPE_BF16 ? K1Shape<1>::CW : K1Shape<0>::CW;
   rp.tiles_per_row = (n_chunks + tile_chunks - 1) / tile_chunks;
   rp.total_tiles = rows * rp.tiles_per_row;
@@ -420,6 +422,35 @@ __global__ void reset_tree_kernel(int B, int N, int n_max, const int* tail, int*
   const int b = (int)(i / N), u = (int)(i % N);
   tree[i] = u == 0 ? tail[b * n_max + n_max - 1] : -1;
   cand_n[i] = 0;
+}
+
+// After a state import: a drafted node must carry a token of the vocabulary that its parent's candidate list
+// holds (that list is the draft distribution the verification divides by), under a drafted parent.  A node
+// that does not is cleared and counted; candidate counts are clamped to the list's capacity.
+__global__ void validate_state_kernel(int B, int N, int K, int V, const int* parent, int* tree, int* cand_n, const int* cand_id,
+                                      unsigned long long* stats) {
+  const long long i = (long long)blockIdx.x * blockDim.x + threadIdx.x;
+  if (i >= (long long)B * N) return;
+  const int b = (int)(i / N), v = (int)(i % N);
+  int cn = cand_n[i];
+  if (cn < 0 || cn > K) { cn = cn < 0 ? 0 : K; cand_n[i] = cn; }
+  if (v == 0) return;
+  const int tok = tree[i];
+  if (tok < 0) return;
+  const int par = parent[v];
+  const long long pi = (long long)b * N + par;
+  bool ok = tok < V && (par == 0 || tree[pi] >= 0);
+  if (ok) {
+    int pn = cand_n[pi];
+    pn = pn < 0 ? 0 : (pn > K ? K : pn);
+    bool listed = false;
+    for (int t = 0; t < pn; ++t) listed |= cand_id[pi * K + t] == tok;
+    ok = listed;
+  }
+  if (!ok) {
+    tree[i] = -1;
+    atomicAdd(&stats[ST_BAD_TOKENS], 1ull);
+  }
 }
 
 // The records of the last verification as rows for a bulk update: positions past a sequence's accepted
@@ -663,7 +694,8 @@ int stand_row_stats_static(const void* dev_logits, int64_t rows, int32_t V, int3
                            int32_t topk, float* dev_lse, int32_t* dev_ids, float* dev_values, float* dev_probs,
                            void* cu_stream) {
   const size_t need = stand_row_stats_scratch_bytes(rows, V, dtype, topk);
-  if (need == 0) return STAND_E_ARG;
+  // the same argument checks, in the same order, as stand_row_stats: an invalid call is an invalid call at any size
+  if (need == 0 || !dev_logits || !dev_lse || !dev_ids || !dev_values || !dev_probs || !(temperature > 0.0f)) return STAND_E_ARG;
   if (need > (size_t)STAND_STATIC_SCRATCH_BYTES) return STAND_E_TOO_LARGE;
   int dev = -1;
   if (cudaGetDevice(&dev) != cudaSuccess) return STAND_E_CUDA;
@@ -794,6 +826,13 @@ int stand_state_load(stand_ctx* x, const int32_t* dev_tail, const int64_t* dev_l
   cp(x->L.cand_n, dev_cand_n, BN * 4);
   cp(x->L.cand_id, dev_cand_id, BN * c.topk * 4);
   cp(x->L.cand_phi, dev_cand_phi, BN * c.topk * 4);
+  if (rc == STAND_OK) {
+    validate_state_kernel<<<(unsigned)((BN + 255) / 256), 256, 0, st>>>(c.B, c.N, c.topk, c.V, x->topo_parent(), x->at<int>(x->L.tree),
+                                                                       x->at<int>(x->L.cand_n), x->at<int>(x->L.cand_id),
+                                                                       x->at<unsigned long long>(x->L.stats));
+    rc = launch_ok();
+    if (rc == STAND_OK) x->launches += 1;
+  }
   if (rc == STAND_OK) { x->step = step; x->pending = false; x->located = false; }
   return rc;
 }
@@ -886,6 +925,11 @@ int stand_profile_stages(stand_ctx* x, void* const* events) {
 }
 
 uint64_t stand_launch_count(const stand_ctx* x) { return x ? x->launches : 0; }
+
+int stand_set_wait_limit(int64_t polls) {
+  g_empty_wait_limit.store(polls < 0 || polls > (int64_t)SPIN_LIMIT ? SPIN_LIMIT : (unsigned)polls, std::memory_order_relaxed);
+  return STAND_OK;
+}
 
 const char* stand_strerror(int code) {
   switch (code) {

@@ -249,12 +249,13 @@ struct UpdateParams {
   unsigned long long* stats;
 };
 
-// The locate step of one record; called by all lanes of a warp, 8 lanes per record.
-__device__ __forceinline__ void locate_record(const UpdateParams& p, long long row, int n, bool in_range) {
+// The locate step of one record; called by all lanes of a warp, 8 lanes per record.  check_path false: the
+// row is known to lie on its sequence's accepted path (n_path need not have been written yet).
+__device__ __forceinline__ void locate_record(const UpdateParams& p, long long row, int n, bool in_range, bool check_path = true) {
   const int gl = threadIdx.x & (GROUP - 1);
   int key[4] = {-1, -1, -1, -1};
   bool ok = in_range;
-  if (ok && p.n_path) ok = (int)(row % p.width) < p.n_path[row / p.width];
+  if (ok && check_path && p.n_path) ok = (int)(row % p.width) < p.n_path[row / p.width];
   if (ok) {
     for (int i = 0; i < n; ++i) {
       const int t = p.rec_ctx[row * p.n_max + (p.n_max - n + i)];

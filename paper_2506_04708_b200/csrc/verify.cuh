@@ -275,7 +275,8 @@ __device__ __forceinline__ void verify_block(const VerifyParams& p, const int b)
   const double cd = (double)p.c;
 
   pdl_trigger();
-  // ---- phase 0: stage the sequence's state (written before the row pass of this step began) ------------------------------------------
+  // ---- phase 0: stage the sequence's state.  It was written by the previous step, and this block cannot
+  // have been scheduled before that step ended: the row pass releases its dependents only after its own wait ----
   for (int u = tid; u < N; u += K2_THREADS) {
     s_tree[u] = p.tree[(long long)b * N + u];
     s_cn[u] = p.cand_n[(long long)b * N + u];
@@ -402,14 +403,17 @@ __device__ __forceinline__ void verify_block(const VerifyParams& p, const int b)
         const double U = __shfl_sync(FULL, Uj, j & 15);
         const double qx = __shfl_sync(FULL, qh, ix < 0 ? 0 : ix);
         const double px = __shfl_sync(FULL, ph, ix < 0 ? 0 : ix);
+        // A drafted token always comes from its parent's candidate list (stand_state_load clears any that does
+        // not); should one be met all the same, it and its later siblings count as not drafted.
+        if (ix < 0) break;
         if (p.deterministic) {
           // one-hot draft: accept iff U < p~(x); on rejection x loses its mass and the rest is renormalised
-          if (ix < 0 || U * zr < px) { accepted = j; break; }
+          if (U * zr < px) { accepted = j; break; }
           zr -= px;
           if (li == ix) ph = 0.0;
           continue;
         }
-        if (ix < 0 || U * qx * zr < px * qn) { accepted = j; break; }
+        if (U * qx * zr < px * qn) { accepted = j; break; }
         const double a = ph * qn, c2 = qh * zr;
         const double ov = half_sum_d(fmin(a, c2));
         pq *= qn;

@@ -7,6 +7,8 @@ state and the whole N-gram table.  It needs a GPU and the built oracle; one JSON
 
     python tests/long_parity.py --workload cfg3                 # all 8,192 steps
     python tests/long_parity.py --workload cfg5 --steps 128 --peak-mode p80
+
+Every run appends its JSON line to --record (tests/parity_runs.jsonl by default), the tracked record of these runs.
 """
 import argparse
 import json
@@ -28,6 +30,8 @@ def main():
     ap.add_argument("--seed", type=int, default=0)
     ap.add_argument("--check-every", type=int, default=0, help="also compare state and table every so many steps")
     ap.add_argument("--deterministic", action="store_true")
+    ap.add_argument("--record", default=os.path.join(os.path.dirname(os.path.abspath(__file__)), "parity_runs.jsonl"),
+                    help="file the run's JSON line is appended to")
     args = ap.parse_args()
 
     w = inputs.WORKLOADS[args.workload]
@@ -56,12 +60,14 @@ def main():
         "drafting": "deterministic" if args.deterministic else "stochastic",
         "rows_compared": steps * w.B * w.N, "emitted_tokens": loop.emitted_total,
         "acceptance_length": loop.emitted_total / (steps * w.B),
-        "hard_mismatches": len(loop.hard), "tolerated_low_margin": loop.tolerated,
+        "hard_mismatches": len(loop.hard), "tolerated_low_margin": loop.tolerated, "tolerated_by": loop.tolerated_by,
         "state_and_table_differences": len(final), "intermediate_checks": checks,
         "table_contexts": contexts, "drops": st["drops"], "bad_tokens": st["bad_tokens"],
         "wait_timeouts": st["wait_timeouts"], "max_probe": st["max_probe_seen"], "seconds": round(time.time() - t0, 1),
     }
     print(json.dumps(out), flush=True)
+    with open(args.record, "a") as f:
+        f.write(json.dumps(out) + "\n")
     ok = not loop.hard and not final and not any(checks) and st["drops"] == 0 and st["wait_timeouts"] == 0
     sys.exit(0 if ok else 1)
 

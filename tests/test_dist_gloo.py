@@ -95,3 +95,16 @@ def test_record_exchange_keeps_global_sequence_order(tmp_path):
     import torch
     rows = (torch.zeros(2, 3), torch.zeros(2, 5), torch.zeros(2, 5))
     assert sharded.gather_rows(None, rows) is rows
+
+
+def test_bench_starts_its_own_ranks_when_run_without_a_launcher():
+    """`python bench.py --gpus 2` with no launcher environment starts two ranks itself (torch.distributed.run on
+    127.0.0.1) and reports n_gpus = 2.  The reference arm needs no GPU, so this runs here: rank 0 times the
+    oracle and prints the line, rank 1 exits without work."""
+    env = {k: v for k, v in os.environ.items() if k not in ("RANK", "WORLD_SIZE", "LOCAL_RANK", "MASTER_ADDR", "MASTER_PORT")}
+    out = subprocess.run([sys.executable, os.path.join(ROOT, "bench.py"), "--impl", "reference", "--gpus", "2", "--steps", "1",
+                          "--warmup", "0", "--workload", "cfg1"], env=env, capture_output=True, text=True, timeout=600)
+    assert out.returncode == 0, out.stderr[-2000:]
+    lines = [json.loads(l) for l in out.stdout.splitlines() if l.startswith("{")]
+    assert len(lines) == 1
+    assert lines[0]["impl"] == "reference" and lines[0]["n_gpus"] == 2 and lines[0]["value"] > 0

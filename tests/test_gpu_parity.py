@@ -122,8 +122,8 @@ def _run(w, steps, peak_mode, seed=0, check_every=0, **kw):
         assert loop.check_state_and_table() == []
         st = loop.gpu.stats()
         assert st["drops"] == 0 and st["bad_tokens"] == 0 and st["wait_timeouts"] == 0
-        # a handful of low-margin decisions at most
-        assert loop.tolerated <= max(2, steps // 100)
+        # low-margin decisions are rare: a few per ten thousand verified rows at most
+        assert loop.tolerated <= max(2, int(3e-4 * steps * w.B * w.N))
         return loop.emitted_total / (steps * w.B), loop.tolerated, st
     finally:
         loop.close()
@@ -144,11 +144,12 @@ def test_cfg2_window(peak_mode):
 
 @pytest.mark.parametrize("peak_mode", ["add8", "p80"])
 def test_cfg3_window(peak_mode):
-    _run(inputs.WORKLOADS["cfg3"], 10, peak_mode, table_slots=1 << 16, check_every=5)
+    _run(inputs.WORKLOADS["cfg3"], 64, peak_mode, table_slots=1 << 18, check_every=32, device_logits=True)
 
 
-def test_cfg4_window():
-    _run(inputs.WORKLOADS["cfg4"], 5, "p80", table_slots=1 << 16, check_every=5)
+@pytest.mark.parametrize("peak_mode", ["add8", "p80"])
+def test_cfg4_window(peak_mode):
+    _run(inputs.WORKLOADS["cfg4"], 32, peak_mode, table_slots=1 << 18, check_every=16, device_logits=True)
 
 
 def test_cfg5_shape_small_vocab():
@@ -510,6 +511,77 @@ def test_full_table_drops_updates_and_never_hangs():
     assert st["drops"] > 0 and st["inserts"] <= 64
     assert len(g.table_dict()) == st["inserts"]
     g.close()
+
+
+# ------------------------------------------------- steps in flight, failure path
+@pytest.mark.parametrize("shape", ["cfg1", "B4", "B20"])
+def test_back_to_back_steps_equal_synchronised_steps(shape):
+    """200 stand_step calls queued with nothing between them and no host synchronisation, against the same
+    steps run one at a time.  Small grids leave most of the GPU free, so a kernel of the next step that started
+    before the previous step's state was complete would read stale trees, candidate lists or tails here."""
+    torch = _torch()
+    from paper_2506_04708_b200.binding import Stand
+    base = inputs.WORKLOADS["cfg1"]
+    w = {"cfg1": inputs.scaled(base, steps=200), "B4": inputs.scaled(base, B=4, V=4096, steps=200),
+         "B20": inputs.scaled(base, B=20, V=4096, steps=200)}[shape]
+    parent = inputs.topology(w.N, w.D, w.kb)
+    depth = inputs.node_depths(parent)
+    streams = inputs.token_streams(w, 7, 8 + (w.steps + 2) * (w.D + 2))
+    tail = torch.from_numpy(streams[:, 5:8].copy())
+    lens0 = torch.full((w.B,), 8, dtype=torch.int64)
+    mk = lambda: Stand(w.B, w.N, w.V, w.topk, w.order_max, w.dtype, w.T, 7, 1 << 14, parent)
+    # pass 1, one step at a time: the closed loop makes each step's logits from the lengths so far
+    a = mk()
+    a.reset_sequences(tail, lens0)
+    gen = inputs.DeviceLogits(w, streams, depth, 7, pool=2, device=a.dev, peak_mode="p80")
+    logits, want = [], []
+    lens = torch.empty(w.B, dtype=torch.int64, device=a.dev)
+    for s in range(w.steps):
+        a.lens_device(lens)
+        buf = torch.empty((w.B, w.N, w.V), dtype=torch.float32, device=a.dev)
+        gen.make(buf, lens, s)
+        out = a.step(buf)
+        torch.cuda.synchronize()
+        logits.append(buf)
+        want.append([t.clone() for t in out])
+    # pass 2, a fresh context: the same logits, every step writing its own result buffers, nothing else queued
+    b = mk()
+    b.reset_sequences(tail, lens0)
+    i32 = dict(dtype=torch.int32, device=b.dev)
+    got = [(torch.empty((w.B, b.D + 1), **i32), torch.empty(w.B, **i32), torch.empty((w.B, w.N), **i32)) for _ in range(w.steps)]
+    torch.cuda.synchronize()
+    for s in range(w.steps):
+        b.step(logits[s], out=got[s])
+    torch.cuda.synchronize()
+    for s in range(w.steps):
+        for x, y in zip(got[s], want[s]):
+            assert torch.equal(x, y), s
+    assert sum(int(t[1].sum()) for t in want) > 1.2 * w.B * w.steps  # drafts were accepted: the state mattered
+    sa, sb = a.state_dump(), b.state_dump()
+    assert all(np.array_equal(sa[k], sb[k]) for k in sa)
+    assert a.table_dict() == b.table_dict()
+    assert b.stats()["wait_timeouts"] == 0
+    a.close(); b.close()
+
+
+def test_a_wait_that_runs_out_is_reported_and_the_next_call_is_clean():
+    """The streaming kernel's loader is told to give up its first wait at once (nothing has been copied yet, so
+    nothing is in flight): the kernel returns, the failure is reported in-band, and the next call works."""
+    from paper_2506_04708_b200 import binding
+    rng = np.random.default_rng(3)
+    x = (rng.standard_normal((6, 8192)) * 2.5).astype(np.float32)
+    dl = harness.to_device_logits(x)
+    good = [t.cpu().numpy() for t in binding.row_stats(dl, 0.8, 8)]
+    binding.set_wait_limit(0)
+    try:
+        lse, ids, vals, probs = (t.cpu().numpy() for t in binding.row_stats(dl, 0.8, 8))
+    finally:
+        binding.set_wait_limit(-1)
+    assert np.isnan(lse).all() and (ids == -1).all() and (probs == 0).all()
+    again = [t.cpu().numpy() for t in binding.row_stats(dl, 0.8, 8)]
+    assert all(np.array_equal(p, q) for p, q in zip(good, again))
+    olse, oids, _, oprobs, _ = so.row_stats(x[0], float(np.float32(0.8)), 8)
+    assert np.array_equal(again[1][0], oids) and abs(again[0][0] - olse) < 1e-5 * max(1, abs(olse))
 
 
 def test_smoke_entry():

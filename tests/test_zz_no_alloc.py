@@ -7,8 +7,8 @@ that entry point through the C ABI twice in a row (the buffer is shared and keep
 call's contents, so the second call runs on a dirty buffer) and checks both results against
 stand_row_stats, which takes caller-allocated scratch.
 
-The file name makes pytest collect it last, so a run that stops at the first failure has
-already run every other test.  It does not depend on them: it passes in a fresh process too.
+The test does not depend on the order of the run: it passes alone in a fresh process and after
+the other tests (its file is merely collected last).
 """
 import numpy as np
 import pytest
@@ -49,6 +49,28 @@ def test_static_scratch_matches_caller_scratch_twice_in_a_row(dtype):
         _same(again, want, tol)
 
 
+def test_static_calls_leave_device_memory_as_it_is():
+    """With the outputs made beforehand and the buffer's address resolved by a first call, further calls must
+    not change the amount of device memory in use: nothing is allocated or freed, by the library or below it."""
+    import torch
+    from paper_2506_04708_b200 import binding
+    rng = np.random.default_rng(12)
+    rows, V, k = 16, 40000, 10
+    dl = harness.to_device_logits(_case(rng, rows, V, "bf16"))
+    out = (torch.empty(rows, dtype=torch.float32, device="cuda:0"), torch.empty((rows, k), dtype=torch.int32, device="cuda:0"),
+           torch.empty((rows, k), dtype=torch.float32, device="cuda:0"), torch.empty((rows, k), dtype=torch.float32, device="cuda:0"))
+    want = binding.row_stats(dl, 0.9, k)
+    binding.row_stats_static(dl, 0.9, k, out=out)  # the first call on this device resolves the buffer's address
+    torch.cuda.synchronize()
+    free_before, total = torch.cuda.mem_get_info()
+    for _ in range(5):
+        binding.row_stats_static(dl, 0.9, k, out=out)
+    torch.cuda.synchronize()
+    free_after, _ = torch.cuda.mem_get_info()
+    assert free_after == free_before
+    _same(out, want, 4e-3)
+
+
 def test_static_scratch_refuses_what_does_not_fit():
     import torch
     from paper_2506_04708_b200 import binding
@@ -61,3 +83,10 @@ def test_static_scratch_refuses_what_does_not_fit():
                                               *(t.data_ptr() for t in out), None)
     assert rc == -5
     assert b"built-in scratch" in binding.lib().stand_strerror(rc)
+    # an invalid call is reported as such whatever its size: the argument checks come first
+    rc = binding.lib().stand_row_stats_static(dl.data_ptr(), rows, V, binding.DTYPE_BF16, 0.0, k,
+                                              *(t.data_ptr() for t in out), None)
+    assert rc == -1
+    rc = binding.lib().stand_row_stats_static(dl.data_ptr(), rows, V, binding.DTYPE_BF16, 1.0, k, None,
+                                              *(t.data_ptr() for t in out[1:]), None)
+    assert rc == -1
