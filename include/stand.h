@@ -142,6 +142,13 @@ int stand_ngram_update_bulk(stand_ctx* ctx, const int32_t* dev_ctx, const int32_
  * table of one context that held all the sequences.  STAND_E_STATE without a pending verification. */
 int stand_export_records(stand_ctx* ctx, int32_t* dev_ctx, int32_t* dev_ids, float* dev_probs, void* cu_stream);
 
+/* The same exchange with one buffer per context: row r of dev_rows [B*(D+1), order_max + 2*topk] int32 holds the
+ * context window, then the ids, then the probabilities (float bit patterns) of row r as stand_export_records
+ * writes them, so the rows of all contexts travel in ONE gather; stand_ngram_update_packed applies M such rows
+ * in row order, exactly as stand_ngram_update_bulk applies the three arrays. */
+int stand_export_records_packed(stand_ctx* ctx, int32_t* dev_rows, void* cu_stream);
+int stand_ngram_update_packed(stand_ctx* ctx, const int32_t* dev_rows, int64_t M, void* cu_stream);
+
 /* Drops the pending verification's own update (its rows reach the tables through
  * stand_ngram_update_bulk instead).  Host only.  STAND_E_STATE if no verification is pending. */
 int stand_skip_update(stand_ctx* ctx);
@@ -154,7 +161,11 @@ int stand_skip_update(stand_ctx* ctx);
  * NULL) and keeps the tree and the candidate lists for the next verification. */
 int stand_draft_tree(stand_ctx* ctx, int32_t* dev_tree_tokens, void* cu_stream);
 
-/* verify -> update -> draft on one stream, no host synchronisation: two kernel launches for up to 16
+/* All kernels of the hot path are launched with programmatic stream serialisation: each may be scheduled while
+ * the kernel before it in the stream is draining, and stops (griddepcontrol.wait) before it reads anything that
+ * kernel may have written, whichever kernel it is; the stage calls above therefore chain like the fused step.
+ *
+ * verify -> update -> draft on one stream, no host synchronisation: two kernel launches for up to 16
  * sequences (the row pass, then verification, update and drafting in one block, or in one thread-block
  * cluster with a block per sequence), four for larger batches. */
 int stand_step(stand_ctx* ctx, const void* dev_logits, int32_t* dev_emitted, int32_t* dev_n_emitted,

@@ -17,7 +17,8 @@ DTYPE_F32, DTYPE_BF16 = 0, 1
 
 EXPORTS = [
     "stand_workspace_bytes", "stand_init", "stand_destroy", "stand_reset_sequences", "stand_verify_tree",
-    "stand_ngram_update", "stand_ngram_update_bulk", "stand_export_records", "stand_skip_update", "stand_draft_tree", "stand_step", "stand_step_host",
+    "stand_ngram_update", "stand_ngram_update_bulk", "stand_export_records", "stand_export_records_packed",
+    "stand_ngram_update_packed", "stand_skip_update", "stand_draft_tree", "stand_step", "stand_step_host",
     "stand_row_stats_scratch_bytes", "stand_row_stats", "stand_row_stats_static", "stand_get_stats",
     "stand_last_path", "stand_tree_depth", "stand_table_dump", "stand_table_load", "stand_state_dump",
     "stand_state_load", "stand_profile_row_pass", "stand_profile_stages", "stand_node_accepts", "stand_prune_tree",
@@ -69,6 +70,10 @@ def lib():
     L.stand_ngram_update_bulk.argtypes = [vp, vp, vp, vp, i64, vp]
     L.stand_export_records.argtypes = [vp, vp, vp, vp, vp]
     L.stand_export_records.restype = C.c_int
+    L.stand_export_records_packed.argtypes = [vp, vp, vp]
+    L.stand_export_records_packed.restype = C.c_int
+    L.stand_ngram_update_packed.argtypes = [vp, vp, i64, vp]
+    L.stand_ngram_update_packed.restype = C.c_int
     L.stand_skip_update.argtypes = [vp]
     L.stand_skip_update.restype = C.c_int
     L.stand_draft_tree.argtypes = [vp, vp, vp]
@@ -228,6 +233,23 @@ class Stand:
         _check(lib().stand_export_records(self.h, _ptr(ctx), _ptr(ids), _ptr(probs), _stream(stream)),
                "stand_export_records")
         return ctx, ids, probs
+
+    def export_records_packed(self, out=None, stream=None):
+        """The same rows in one int32 tensor [B*(D+1), order_max + 2*topk]: context, ids, probabilities (as bits)."""
+        t = self.torch
+        if out is None:
+            out = t.empty((self.B * (self.D + 1), self.n_max + 2 * self.K), dtype=t.int32, device=self.dev)
+        _check(lib().stand_export_records_packed(self.h, _ptr(out), _stream(stream)), "stand_export_records_packed")
+        return out
+
+    def ngram_update_packed(self, rows, stream=None):
+        """Applies packed rows (as export_records_packed writes them, of any number of contexts) in row order.
+        Does not wait for the kernels: `rows` is kept alive until the next such call."""
+        assert rows.is_cuda and rows.dtype == self.torch.int32 and rows.is_contiguous()
+        assert rows.shape[-1] == self.n_max + 2 * self.K
+        _check(lib().stand_ngram_update_packed(self.h, _ptr(rows), rows.numel() // rows.shape[-1], _stream(stream)),
+               "stand_ngram_update_packed")
+        self._bulk_keep = rows
 
     def skip_update(self):
         _check(lib().stand_skip_update(self.h), "stand_skip_update")

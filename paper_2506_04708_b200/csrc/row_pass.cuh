@@ -341,6 +341,45 @@ __global__ void __launch_bounds__((CW + 1) * 32, CTAS) row_pass_kernel(const Row
   }
 }
 
+// Small launches: every chunk is read by a warp of its own, straight from global memory with 16-byte loads
+// (same alignment requirement as the streaming kernel).  While the whole launch fits the GPU's resident warps a
+// couple of times over, all its loads are in flight at once and the pass costs little more than one memory
+// round trip plus the transfer, where the streaming kernel's few blocks would still be filling their rings.
+#ifndef STAND_DIRECT_WAVES
+#define STAND_DIRECT_WAVES 2  // launches of up to this many waves of resident warps take the direct kernel
+#endif
+constexpr int DIRECT_WARPS = 8;           // warps (chunks) per block of the direct kernel
+constexpr int DIRECT_WARPS_PER_SM = 48;   // resident at its register use
+
+__device__ __forceinline__ uint4 load_stream16(const void* p) {
+  uint4 v;
+  asm volatile("ld.global.nc.L1::no_allocate.v4.u32 {%0, %1, %2, %3}, [%4];" : "=r"(v.x), "=r"(v.y), "=r"(v.z), "=r"(v.w) : "l"(p));
+  return v;
+}
+
+template <int DT>
+__global__ void __launch_bounds__(DIRECT_WARPS * 32) row_pass_direct_kernel(const RowPassParams p) {
+  using TR = ElemTraits<DT>;
+  constexpr int VEC = TR::VEC, NV = CHUNK / (32 * VEC);
+  const int lane = threadIdx.x & 31;
+  const long long unit = (long long)blockIdx.x * DIRECT_WARPS + (threadIdx.x >> 5);
+  pdl_wait();     // chained after the previous step: nothing is read or written before that step has ended
+  pdl_trigger();  // and only then may the next kernel of this step be scheduled (see the streaming kernel)
+  if (unit >= p.rows * p.n_chunks) return;
+  const long long row = unit / p.n_chunks;
+  const int chunk = (int)(unit - row * p.n_chunks);
+  const char* src = (const char*)p.logits + ((size_t)row * (size_t)p.V + (size_t)chunk * CHUNK) * TR::ESIZE;
+  uint4 v[NV];
+#pragma unroll
+  for (int k = 0; k < NV; ++k) {  // V is a multiple of the vector length: a vector lies inside the row or past it
+    const int e = (k * 32 + lane) * VEC;
+    v[k] = chunk * CHUNK + e < p.V ? load_stream16(src + (size_t)e * TR::ESIZE)
+                                   : make_uint4(TR::NEG_INF_WORD, TR::NEG_INF_WORD, TR::NEG_INF_WORD, TR::NEG_INF_WORD);
+  }
+  const float2 r = reduce_chunk<DT, NV>(v, p.c);
+  if (lane == 0) store_pair_keep(p.pairs + unit, r, l2_evict_last_policy());
+}
+
 // Fallback for rows that are not 16-byte aligned: one warp per (row, chunk), scalar loads.
 template <int DT>
 __global__ void __launch_bounds__(256) row_pass_plain_kernel(const RowPassParams p) {

@@ -190,6 +190,17 @@ int launch_row_pass(const void* logits, long long rows, int V, int dtype, int n_
     int sms = 0;
     const int rc = prepare_device(&sms);
     if (rc) return rc;
+    const long long units = rows * n_chunks;
+    if (units <= (long long)STAND_DIRECT_WAVES * DIRECT_WARPS_PER_SM * sms) {  // small: one warp per chunk, everything in flight at once
+      const unsigned blocks = (unsigned)((units + DIRECT_WARPS - 1) / DIRECT_WARPS);
+      if (chain) {
+        if (dtype == STAND_DTYPE_BF16) return launch_dependent(row_pass_direct_kernel<1>, blocks, DIRECT_WARPS * 32u, st, rp);
+        return launch_dependent(row_pass_direct_kernel<0>, blocks, DIRECT_WARPS * 32u, st, rp);
+      }
+      if (dtype == STAND_DTYPE_BF16) row_pass_direct_kernel<1><<<blocks, DIRECT_WARPS * 32, 0, st>>>(rp);
+      else row_pass_direct_kernel<0><<<blocks, DIRECT_WARPS * 32, 0, st>>>(rp);
+      return launch_ok();
+    }
     const long long want = (long long)K1_CTAS * sms;  // each CTA walks a contiguous range of tiles
     const unsigned grid = (unsigned)(rp.total_tiles < want ? rp.total_tiles : want);
     if (chain) {  // may be scheduled while the previous step's last kernel drains; waits for it before any access
@@ -271,11 +282,13 @@ bool cluster_tail_fits(int B, size_t smem) {
 }
 
 UpdateParams update_params(stand_ctx* x, long long n_rows, const int* ctxw, const int* ids, const float* probs,
-                           const int* n_path, int width) {
+                           const int* n_path, int width, int packed_stride = 0) {
   const stand_config& c = x->cfg;
   UpdateParams u;
   u.table = x->at<Slot>(x->L.table); u.mask = c.table_slots - 1; u.max_probe = x->max_probe; u.V = c.V; u.K = c.topk;
   u.n_max = c.order_max; u.n_rows = n_rows; u.rec_ctx = ctxw; u.rec_ids = ids; u.rec_p = probs; u.n_path = n_path;
+  u.ctx_stride = packed_stride ? packed_stride : c.order_max;
+  u.item_stride = packed_stride ? packed_stride : c.topk;
   u.width = width; u.rec_slot = x->at<uint32_t>(x->L.rec_slot); u.stats = x->at<unsigned long long>(x->L.stats);
   return u;
 }
@@ -327,15 +340,15 @@ int run_verify(stand_ctx* x, const void* logits, int32_t* emitted, int32_t* n_em
   if (x->ev_before) cudaEventRecord(x->ev_before, st);
   if (x->ev_stage[0]) cudaEventRecord(x->ev_stage[0], st);
   int rc = launch_row_pass(logits, (long long)c.B * c.N, c.V, c.dtype, x->d.n_chunks, x->c, x->at<float2>(x->L.pairs),
-                           x->at<int>(x->L.status), st, fuse_locate && !x->ev_before && !x->ev_stage[0]);
+                           x->at<int>(x->L.status), st, !x->ev_before && !x->ev_stage[0]);
   if (rc) return rc;
   if (x->ev_after) cudaEventRecord(x->ev_after, st);
   if (x->ev_stage[1]) cudaEventRecord(x->ev_stage[1], st);
   x->launches += 1;
   x->step += 1;  // the tree drafted in step s-1 is verified in step s
   const VerifyParams v = verify_params(x, logits, emitted, n_emitted, fuse_locate);
-  // inside a fused step (and with no timing events between the launches) the kernels chain programmatically
-  const bool chain = fuse_locate && !x->ev_after && !x->ev_stage[1];
+  // with no timing events between the launches the kernels chain programmatically
+  const bool chain = !x->ev_after && !x->ev_stage[1];
   const size_t vsm = verify_smem_bytes(c.N);
   if (chain) rc = launch_dependent(verify_kernel, (unsigned)c.B, K2_THREADS, st, v, vsm);
   else { verify_kernel<<<c.B, K2_THREADS, vsm, st>>>(v); rc = launch_ok(); }
@@ -350,14 +363,18 @@ int run_verify(stand_ctx* x, const void* logits, int32_t* emitted, int32_t* n_em
 int run_update_rows(stand_ctx* x, const UpdateParams& u, bool located, cudaStream_t st) {
   const long long n_rec = u.n_rows * u.n_max;
   int rc;
+  // both stages stop (griddepcontrol.wait) before they read anything, so they may be scheduled while the kernel
+  // before them in the stream drains, whichever kernel that is
+  const bool chain = !x->ev_stage[2];
   if (!located) {
-    update_locate_kernel<<<(unsigned)((n_rec * GROUP + 255) / 256), 256, 0, st>>>(u);
-    rc = launch_ok();
+    const unsigned locate_blocks = (unsigned)((n_rec * GROUP + 255) / 256);
+    if (chain) rc = launch_dependent(update_locate_kernel, locate_blocks, 256u, st, u);
+    else { update_locate_kernel<<<locate_blocks, 256, 0, st>>>(u); rc = launch_ok(); }
     if (rc) return rc;
     x->launches += 1;
   }
   const unsigned apply_blocks = (unsigned)((n_rec + APPLY_WARPS - 1) / APPLY_WARPS);
-  if (located && !x->ev_stage[2]) rc = launch_dependent(update_apply_kernel, apply_blocks, APPLY_WARPS * 32, st, u);
+  if (chain) rc = launch_dependent(update_apply_kernel, apply_blocks, APPLY_WARPS * 32, st, u);
   else { update_apply_kernel<<<apply_blocks, APPLY_WARPS * 32, 0, st>>>(u); rc = launch_ok(); }
   if (rc) return rc;
   x->launches += 1;
@@ -455,19 +472,42 @@ __global__ void validate_state_kernel(int B, int N, int K, int V, const int* par
 
 // The records of the last verification as rows for a bulk update: positions past a sequence's accepted
 // path get an all -1 context (a bulk update skips such a row), ids -1 and probabilities 0.
-__global__ void export_records_kernel(int B, int W, int n_max, int K, const int* n_path, const int* rec_ctx, const int* rec_ids,
-                                      const float* rec_p, int* out_ctx, int* out_ids, float* out_p) {
+struct ExportParams {
+  int B, W, n_max, K;
+  const int* n_path;
+  const int* rec_ctx;
+  const int* rec_ids;
+  const float* rec_p;
+  int* out_ctx;
+  int* out_ids;
+  float* out_p;
+  int ctx_stride, item_stride;
+};
+
+// Output rows are ctx_stride / item_stride words apart (n_max and K for three separate arrays, the row length for
+// packed rows).
+__global__ void export_records_entry(const ExportParams q) {
+  const int B = q.B, W = q.W, n_max = q.n_max, K = q.K, ctx_stride = q.ctx_stride, item_stride = q.item_stride;
+  const int* n_path = q.n_path;
+  const int* rec_ctx = q.rec_ctx;
+  const int* rec_ids = q.rec_ids;
+  const float* rec_p = q.rec_p;
+  int* out_ctx = q.out_ctx;
+  int* out_ids = q.out_ids;
+  float* out_p = q.out_p;
+  pdl_trigger();
+  pdl_wait();  // the records come from the verification kernel before this one
   const long long i = (long long)blockIdx.x * blockDim.x + threadIdx.x;  // one thread per (row, entry)
   const int per_row = n_max + K;
   if (i >= (long long)B * W * per_row) return;
   const long long row = i / per_row;
   const int e = (int)(i - row * per_row);
   const bool live = (int)(row % W) < n_path[row / W];
-  if (e < n_max) out_ctx[row * n_max + e] = live ? rec_ctx[row * n_max + e] : -1;
+  if (e < n_max) out_ctx[row * ctx_stride + e] = live ? rec_ctx[row * n_max + e] : -1;
   else {
     const int k = e - n_max;
-    out_ids[row * K + k] = live ? rec_ids[row * K + k] : -1;
-    out_p[row * K + k] = live ? rec_p[row * K + k] : 0.0f;
+    out_ids[row * item_stride + k] = live ? rec_ids[row * K + k] : -1;
+    out_p[row * item_stride + k] = live ? rec_p[row * K + k] : 0.0f;
   }
 }
 
@@ -594,20 +634,46 @@ int stand_ngram_update_bulk(stand_ctx* x, const int32_t* dev_ctx, const int32_t*
   return STAND_OK;
 }
 
-int stand_export_records(stand_ctx* x, int32_t* dev_ctx, int32_t* dev_ids, float* dev_probs, void* cu_stream) {
-  if (!x || !dev_ctx || !dev_ids || !dev_probs) return STAND_E_ARG;
+static int export_records(stand_ctx* x, int32_t* out_ctx, int32_t* out_ids, float* out_p, int ctx_stride, int item_stride,
+                          cudaStream_t st) {
   if (!x->pending) return STAND_E_STATE;
-  cudaStream_t st = (cudaStream_t)cu_stream;
   x->last_stream = st;
   const stand_config& c = x->cfg;
   const int W = x->d.D + 1;
   const long long n = (long long)c.B * W * (c.order_max + c.topk);
-  export_records_kernel<<<(unsigned)((n + 255) / 256), 256, 0, st>>>(c.B, W, c.order_max, c.topk, x->at<int>(x->L.n_path),
-                                                                     x->at<int>(x->L.rec_ctx), x->at<int>(x->L.rec_ids),
-                                                                     x->at<float>(x->L.rec_p), dev_ctx, dev_ids, dev_probs);
-  const int rc = launch_ok();
+  ExportParams e;
+  e.B = c.B; e.W = W; e.n_max = c.order_max; e.K = c.topk; e.n_path = x->at<int>(x->L.n_path);
+  e.rec_ctx = x->at<int>(x->L.rec_ctx); e.rec_ids = x->at<int>(x->L.rec_ids); e.rec_p = x->at<float>(x->L.rec_p);
+  e.out_ctx = out_ctx; e.out_ids = out_ids; e.out_p = out_p; e.ctx_stride = ctx_stride; e.item_stride = item_stride;
+  const int rc = launch_dependent(export_records_entry, (unsigned)((n + 255) / 256), 256u, st, e);
   if (rc == STAND_OK) x->launches += 1;
   return rc;
+}
+
+int stand_export_records(stand_ctx* x, int32_t* dev_ctx, int32_t* dev_ids, float* dev_probs, void* cu_stream) {
+  if (!x || !dev_ctx || !dev_ids || !dev_probs) return STAND_E_ARG;
+  return export_records(x, dev_ctx, dev_ids, dev_probs, x->cfg.order_max, x->cfg.topk, (cudaStream_t)cu_stream);
+}
+
+int stand_export_records_packed(stand_ctx* x, int32_t* dev_rows, void* cu_stream) {
+  if (!x || !dev_rows) return STAND_E_ARG;
+  const int n = x->cfg.order_max, K = x->cfg.topk, stride = n + 2 * K;
+  return export_records(x, dev_rows, dev_rows + n, reinterpret_cast<float*>(dev_rows + n + K), stride, stride, (cudaStream_t)cu_stream);
+}
+
+int stand_ngram_update_packed(stand_ctx* x, const int32_t* dev_rows, int64_t M, void* cu_stream) {
+  if (!x || M < 0 || (M > 0 && !dev_rows)) return STAND_E_ARG;
+  cudaStream_t st = (cudaStream_t)cu_stream;
+  x->last_stream = st;
+  const int n = x->cfg.order_max, K = x->cfg.topk, stride = n + 2 * K;
+  for (int64_t at = 0; at < M; at += BULK_ROWS) {
+    const long long rows = M - at < BULK_ROWS ? M - at : BULK_ROWS;
+    const int32_t* base = dev_rows + at * stride;
+    const int rc = run_update_rows(x, update_params(x, rows, base, base + n, reinterpret_cast<const float*>(base + n + K), nullptr, 1,
+                                                    stride), false, st);
+    if (rc) return rc;
+  }
+  return STAND_OK;
 }
 
 int stand_skip_update(stand_ctx* x) {
@@ -620,7 +686,7 @@ int stand_skip_update(stand_ctx* x) {
 int stand_draft_tree(stand_ctx* x, int32_t* dev_tree_tokens, void* cu_stream) {
   if (!x) return STAND_E_ARG;
   x->last_stream = (cudaStream_t)cu_stream;
-  return run_draft(x, dev_tree_tokens, false, (cudaStream_t)cu_stream);
+  return run_draft(x, dev_tree_tokens, true, (cudaStream_t)cu_stream);
 }
 
 int stand_step(stand_ctx* x, const void* dev_logits, int32_t* dev_emitted, int32_t* dev_n_emitted, int32_t* dev_tree_tokens,

@@ -240,9 +240,10 @@ struct UpdateParams {
   unsigned long long mask;
   int max_probe, V, K, n_max;
   long long n_rows;
-  const int* rec_ctx;   // [n_rows, n_max]
-  const int* rec_ids;   // [n_rows, K]
-  const float* rec_p;   // [n_rows, K]
+  const int* rec_ctx;   // [n_rows, n_max]   rows ctx_stride words apart
+  const int* rec_ids;   // [n_rows, K]       rows item_stride words apart
+  const float* rec_p;   // [n_rows, K]       rows item_stride words apart
+  int ctx_stride, item_stride;  // n_max and K for separate arrays; the row length for rows packed as (ctx, ids, probs)
   const int* n_path;    // [n_rows / width] or null (all rows count)
   int width;            // rows per sequence when n_path is given
   uint32_t* rec_slot;   // [n_max, n_rows]
@@ -258,7 +259,7 @@ __device__ __forceinline__ void locate_record(const UpdateParams& p, long long r
   if (ok && check_path && p.n_path) ok = (int)(row % p.width) < p.n_path[row / p.width];
   if (ok) {
     for (int i = 0; i < n; ++i) {
-      const int t = p.rec_ctx[row * p.n_max + (p.n_max - n + i)];
+      const int t = p.rec_ctx[row * p.ctx_stride + (p.n_max - n + i)];
       if (t < 0) ok = false;  // context shorter than n: this order is skipped
       else if (t >= p.V) {
         ok = false;
@@ -278,6 +279,8 @@ __device__ __forceinline__ void locate_record(const UpdateParams& p, long long r
 }
 
 __global__ void __launch_bounds__(256) update_locate_kernel(const UpdateParams p) {
+  pdl_trigger();
+  pdl_wait();  // the rows may come from the kernel before this one
   const long long g = ((long long)blockIdx.x * blockDim.x + threadIdx.x) / GROUP;  // record index
   const bool in_range = g < p.n_rows * p.n_max;
   const long long row = in_range ? g / p.n_max : 0;
@@ -357,8 +360,8 @@ __device__ __forceinline__ void load_fresh(const UpdateParams& p, long long i, i
   fid = -1;
   fp = 0.0f;
   if (lane >= 16 && lane < 16 + p.K) {
-    fid = p.rec_ids[i * p.K + (lane - 16)];
-    fp = p.rec_p[i * p.K + (lane - 16)];
+    fid = p.rec_ids[i * p.item_stride + (lane - 16)];
+    fp = p.rec_p[i * p.item_stride + (lane - 16)];
   }
 }
 

@@ -2,7 +2,7 @@
 
 Each rank holds a contiguous block of the batch (its context is created with seq_base = the global index
 of its first sequence) and a full copy of the table.  A step is: verify locally, exchange the accepted
-rows (Sec. 4.1's update records: a few KB per sequence, never the logits), apply the rows of ALL ranks in
+rows (Sec. 4.1's update records: a few KB per sequence, never the logits; one gather of one packed buffer), apply the rows of ALL ranks in
 global sequence order, draft locally.  Every copy of the table then equals the table of one context that
 held the whole batch, and so does every draft.
 
@@ -12,23 +12,21 @@ import torch
 
 
 def concat_rows(parts):
-    """parts: per shard (ctx, ids, probs), in the order of their seq_base -> one (ctx, ids, probs)."""
-    return tuple(torch.cat([p[i] for p in parts], dim=0) for i in range(3))
+    """parts: per shard packed rows [rows, order_max + 2*topk], in the order of their seq_base -> one tensor."""
+    return torch.cat(list(parts), dim=0)
 
 
-def gather_rows(dist, rows):
-    """All ranks' (ctx, ids, probs) concatenated in rank order.  Every rank must pass the same shapes (same
-    sequences per rank, same tree), and rank r must hold the sequences before those of rank r + 1."""
+def gather_rows(dist, rows, out=None):
+    """All ranks' packed rows concatenated in rank order, with ONE collective.  Every rank must pass the same
+    shape (same sequences per rank, same tree), and rank r must hold the sequences before those of rank r + 1."""
     if dist is None:
         return rows
     world = dist.get_world_size()
-    out = []
-    for t in rows:
-        t = t.contiguous()
-        buf = torch.empty((world * t.shape[0],) + tuple(t.shape[1:]), dtype=t.dtype, device=t.device)
-        dist.all_gather(list(buf.chunk(world, dim=0)), t)  # rank r's rows land in the r-th block of buf
-        out.append(buf)
-    return tuple(out)
+    rows = rows.contiguous()
+    if out is None:
+        out = torch.empty((world * rows.shape[0],) + tuple(rows.shape[1:]), dtype=rows.dtype, device=rows.device)
+    dist.all_gather_into_tensor(out, rows)  # rank r's rows land in the r-th block
+    return out
 
 
 class ShardedStand:
@@ -37,21 +35,25 @@ class ShardedStand:
     def __init__(self, stand, dist=None):
         self.stand = stand
         self.dist = dist
+        self._mine = self._all = None
         if dist is not None:
             assert stand.seq_base == dist.get_rank() * stand.B, "rank r holds sequences [r * B, (r + 1) * B)"
+            rows, width = stand.B * (stand.D + 1), stand.n_max + 2 * stand.K
+            self._mine = torch.empty((rows, width), dtype=torch.int32, device=stand.dev)
+            self._all = torch.empty((dist.get_world_size() * rows, width), dtype=torch.int32, device=stand.dev)
 
     def verify(self, logits):
-        """Local verification; returns this rank's rows for the exchange."""
+        """Local verification; returns this rank's packed rows for the exchange."""
         self.stand.verify_tree(logits)
-        rows = self.stand.export_records()
+        rows = self.stand.export_records_packed(out=self._mine)
         self.stand.skip_update()
         return rows
 
     def finish(self, all_rows):
         """Applies the rows of all ranks (already in global sequence order) and drafts the next tree."""
-        self.stand.ngram_update_bulk(*all_rows, sync=False)
+        self.stand.ngram_update_packed(all_rows)
         return self.stand.draft_tree()
 
     def step(self, logits):
         rows = self.verify(logits)
-        return self.finish(gather_rows(self.dist, rows))
+        return self.finish(gather_rows(self.dist, rows, self._all))

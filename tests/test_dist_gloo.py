@@ -71,30 +71,32 @@ def _exchange_worker(rank, world, port, out_dir):
     ctx = torch.stack([seq, pos, seq * 100 + pos], dim=1).to(torch.int32)
     ids = (seq * 1000 + pos * 10).to(torch.int32)[:, None] + torch.arange(K, dtype=torch.int32)[None, :]
     probs = (seq.double() + pos.double() / 10)[:, None].float().repeat(1, K)
-    g_ctx, g_ids, g_probs = sharded.gather_rows(d, (ctx, ids, probs))
-    np.savez(os.path.join(out_dir, f"x{rank}.npz"), ctx=g_ctx.numpy(), ids=g_ids.numpy(), probs=g_probs.numpy())
+    rows = torch.cat([ctx, ids, probs.view(torch.int32)], dim=1)   # the packed layout: context, ids, probability bits
+    got = sharded.gather_rows(d, rows)
+    np.save(os.path.join(out_dir, f"x{rank}.npy"), got.numpy())
     sd.barrier(d)
     d.destroy_process_group()
 
 
 def test_record_exchange_keeps_global_sequence_order(tmp_path):
     """The update rows of all ranks arrive on every rank in (sequence, path position) order of the whole batch: the
-    order in which one context holding the whole batch applies them."""
+    order in which one context holding the whole batch applies them.  One collective moves everything."""
     import numpy as np
     world, port = 2, 31000 + os.getpid() % 2000
     mp.spawn(_exchange_worker, args=(world, port, str(tmp_path)), nprocs=world, join=True)
-    r = [np.load(tmp_path / f"x{k}.npz") for k in range(world)]
-    for k in ("ctx", "ids", "probs"):
-        assert np.array_equal(r[0][k], r[1][k])
-    ctx = r[0]["ctx"]
-    assert ctx.shape == (2 * 3 * 4, 3)
+    r = [np.load(tmp_path / f"x{k}.npy") for k in range(world)]
+    assert np.array_equal(r[0], r[1])
+    rows = r[0]
+    assert rows.shape == (2 * 3 * 4, 3 + 2 * 5)
+    ctx, ids, probs = rows[:, :3], rows[:, 3:8], rows[:, 8:].copy().view(np.float32)
     order = ctx[:, 0] * 4 + ctx[:, 1]
     assert np.array_equal(order, np.arange(24))
-    assert np.array_equal(r[0]["ids"][:, 0], ctx[:, 0] * 1000 + ctx[:, 1] * 10)
+    assert np.array_equal(ids[:, 0], ctx[:, 0] * 1000 + ctx[:, 1] * 10)
+    assert np.allclose(probs[:, 0], ctx[:, 0] + ctx[:, 1] / 10)
     # no group: the rows pass through untouched
     import torch
-    rows = (torch.zeros(2, 3), torch.zeros(2, 5), torch.zeros(2, 5))
-    assert sharded.gather_rows(None, rows) is rows
+    one = torch.zeros(2, 13, dtype=torch.int32)
+    assert sharded.gather_rows(None, one) is one
 
 
 def test_bench_starts_its_own_ranks_when_run_without_a_launcher():

@@ -42,6 +42,28 @@ def test_row_stats_matches_oracle(dtype, V):
         assert np.allclose(probs[r, :kk], oprobs[:kk], rtol=tol, atol=1e-30)
 
 
+@pytest.mark.parametrize("dtype,V", [("bf16", 151936), ("f32", 128256), ("bf16", 40008)])
+def test_row_stats_large_launch_takes_the_streaming_kernel(dtype, V):
+    """Launches of more than a couple of waves of chunks go through the bulk-copy ring (smaller ones are read
+    directly, one warp per chunk): enough rows to be there, sampled rows against the oracle."""
+    from paper_2506_04708_b200 import binding
+    torch = _torch()
+    rows, k, T = (130 if V > 100000 else 420), 10, 0.7
+    g = torch.Generator(device="cuda:0").manual_seed(V)
+    x = torch.randn((rows, V), generator=g, device="cuda:0") * 2.5
+    x[torch.arange(rows), torch.randint(0, V, (rows,), generator=g, device="cuda:0")] += 8.0
+    dl = x.to(torch.bfloat16) if dtype == "bf16" else x
+    host = dl.cpu()
+    raw = host.view(torch.int16).numpy().view(np.uint16) if dtype == "bf16" else host.numpy()
+    lse, ids, vals, probs = (t.cpu().numpy() for t in binding.row_stats(dl, T, k))
+    tol = harness.value_tol(inputs.DTYPE_BF16 if dtype == "bf16" else inputs.DTYPE_F32)
+    for r in list(range(0, rows, 13)) + [rows - 1]:
+        olse, oids, ovals, oprobs, _ = so.row_stats(raw[r], float(np.float32(T)), k)
+        assert np.array_equal(ids[r], oids), (r, ids[r], oids)
+        assert abs(lse[r] - olse) <= 1e-5 * max(1.0, abs(olse))
+        assert np.allclose(probs[r], oprobs, rtol=tol, atol=1e-30)
+
+
 def test_row_stats_unaligned_rows_and_many_rows():
     from paper_2506_04708_b200 import binding
     torch = _torch()
@@ -569,7 +591,7 @@ def test_a_wait_that_runs_out_is_reported_and_the_next_call_is_clean():
     nothing is in flight): the kernel returns, the failure is reported in-band, and the next call works."""
     from paper_2506_04708_b200 import binding
     rng = np.random.default_rng(3)
-    x = (rng.standard_normal((6, 8192)) * 2.5).astype(np.float32)
+    x = (rng.standard_normal((400, 40000)) * 2.5).astype(np.float32)  # large enough for the streaming kernel
     dl = harness.to_device_logits(x)
     good = [t.cpu().numpy() for t in binding.row_stats(dl, 0.8, 8)]
     binding.set_wait_limit(0)
