@@ -55,20 +55,21 @@ __device__ __noinline__ int gumbel_rank_double(bool valid, int id, float phi, ui
   return rank;
 }
 
-// The next tree of sequence b by one block of K4_THREADS threads.  WAIT: stop (griddepcontrol.wait) before the first
+// The next tree of sequence b by one block of NT threads (one warp per parent node of a level: trees with more
+// than NT / 32 parents on a level take several rounds there).  WAIT: stop (griddepcontrol.wait) before the first
 // read of what the previous kernel wrote; false when the caller has already ordered itself after that kernel.
-template <bool WAIT>
+template <bool WAIT, int NT = K4_THREADS>
 __device__ __forceinline__ void draft_block(const DraftParams& p, const int b) {
   __shared__ int s_tok[NODES_MAX], s_parent[NODES_MAX], s_fc[NODES_MAX], s_nch[NODES_MAX];
   __shared__ int s_tail[ORDER_MAX], s_level[DEPTH_MAX + 2];
-  __shared__ Slot s_slot[K4_THREADS / 32];  // per warp: the slot that won the lookup
-  __shared__ float s_g[K4_THREADS / 32][KMAX];  // per warp: the candidates' perturbed scores and ids
-  __shared__ int s_gid[K4_THREADS / 32][KMAX];
+  __shared__ Slot s_slot[NT / 32];  // per warp: the slot that won the lookup
+  __shared__ float s_g[NT / 32][KMAX];  // per warp: the candidates' perturbed scores and ids
+  __shared__ int s_gid[NT / 32][KMAX];
   const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
   const int N = p.N, K = p.K, n_max = p.n_max;
   pdl_trigger();
   // topology and tail once, with coalesced loads: the level loop below touches shared memory only
-  for (int u = tid; u < N; u += K4_THREADS) {
+  for (int u = tid; u < N; u += NT) {
     s_tok[u] = -1;
     s_parent[u] = p.parent[u];
     s_fc[u] = p.first_child[u];
@@ -83,7 +84,7 @@ __device__ __forceinline__ void draft_block(const DraftParams& p, const int b) {
 
   for (int d = 0; d < p.D; ++d) {
     const int l0 = s_level[d], l1 = s_level[d + 1];
-    for (int u = l0 + warp; u < l1; u += K4_THREADS / 32) {
+    for (int u = l0 + warp; u < l1; u += NT / 32) {
       const int m = s_nch[u];
       const long long row = (long long)b * N + u;
       if (m == 0) { if (lane == 0) p.cand_n[row] = 0; continue; }
@@ -181,8 +182,8 @@ __device__ __forceinline__ void draft_block(const DraftParams& p, const int b) {
     __syncthreads();
   }
   // nodes of the deepest level have no children
-  for (int u = s_level[p.D] + tid; u < N; u += K4_THREADS) p.cand_n[(long long)b * N + u] = 0;
-  for (int u = tid; u < N; u += K4_THREADS) {
+  for (int u = s_level[p.D] + tid; u < N; u += NT) p.cand_n[(long long)b * N + u] = 0;
+  for (int u = tid; u < N; u += NT) {
     const int t = s_tok[u];
     p.tree[(long long)b * N + u] = t;
     if (p.tree_user) p.tree_user[(long long)b * N + u] = t;

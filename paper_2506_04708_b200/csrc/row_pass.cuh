@@ -343,10 +343,12 @@ __global__ void __launch_bounds__((CW + 1) * 32, CTAS) row_pass_kernel(const Row
 
 // Small launches: every chunk is read by a warp of its own, straight from global memory with 16-byte loads
 // (same alignment requirement as the streaming kernel).  While the whole launch fits the GPU's resident warps a
-// couple of times over, all its loads are in flight at once and the pass costs little more than one memory
+// few times over, most of its loads are in flight at once and the pass costs little more than one memory
 // round trip plus the transfer, where the streaming kernel's few blocks would still be filling their rings.
+// Measured alone, back to back (us per launch, streaming / direct): 64 rows of 151,936 bf16 10.2 / 7.0; 128 rows
+// 12.9 / 10.3; 512 rows 29.2 / 28.9; 1,024 rows 50.7 / 55.3: the streaming kernel wins from about ten waves on.
 #ifndef STAND_DIRECT_WAVES
-#define STAND_DIRECT_WAVES 2  // launches of up to this many waves of resident warps take the direct kernel
+#define STAND_DIRECT_WAVES 8  // launches of up to this many waves of resident warps take the direct kernel
 #endif
 constexpr int DIRECT_WARPS = 8;           // warps (chunks) per block of the direct kernel
 constexpr int DIRECT_WARPS_PER_SM = 48;   // resident at its register use

@@ -264,7 +264,7 @@ bool cluster_tail_fits(int B, size_t smem) {
   if (B < 2 || B > TAIL_CLUSTER_MAX) return false;
   cudaLaunchConfig_t cfg = {};
   cfg.gridDim = dim3((unsigned)B);
-  cfg.blockDim = dim3(K2_THREADS);
+  cfg.blockDim = dim3(TAIL_THREADS);
   cfg.dynamicSmemBytes = smem;
   cudaLaunchAttribute attr[1];
   attr[0].id = cudaLaunchAttributeClusterDimension;
@@ -418,8 +418,8 @@ int run_step(stand_ctx* x, const void* logits, int32_t* emitted, int32_t* n_emit
     TailParams t;
     t.v = verify_params(x, logits, emitted, n_emitted, true);
     t.d = draft_params(x, tree_user);
-    if (x->tail_form == 1) rc = launch_dependent(tail_single_kernel, 1u, K2_THREADS, st, t, verify_smem_bytes(c.N));
-    else rc = launch_dependent_cluster(tail_cluster_kernel, (unsigned)c.B, K2_THREADS, st, t, verify_smem_bytes(c.N));
+    if (x->tail_form == 1) rc = launch_dependent(tail_single_kernel, 1u, TAIL_THREADS, st, t, verify_smem_bytes(c.N));
+    else rc = launch_dependent_cluster(tail_cluster_kernel, (unsigned)c.B, TAIL_THREADS, st, t, verify_smem_bytes(c.N));
     if (rc) return rc;
     x->launches += 2;
     x->pending = false;

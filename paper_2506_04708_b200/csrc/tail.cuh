@@ -13,8 +13,13 @@ namespace stand {
 // stage 2 of the update, drafting.  Where the batch form relies on a kernel boundary ("every sequence has
 // located its records", "the table is up to date") this form has a block barrier, or the hardware barrier
 // of the cluster, whose release/acquire pair also orders the blocks' global-memory writes.
-static_assert(K2_THREADS == K4_THREADS && K2_THREADS == APPLY_WARPS * 32, "one block shape for the three stages");
+// The block is TAIL_THREADS wide: its first K2_THREADS threads verify (on a named barrier of their own); the others
+// map the update records to table slots as soon as the walk has emitted its tokens, beside the compression of the
+// accepted rows; all of them then apply the records and draft, where more warps mean fewer rounds (one warp per
+// record, one warp per parent node of a tree level).
+constexpr int TAIL_THREADS = 512;
 constexpr int TAIL_CLUSTER_MAX = 16;  // largest cluster the hardware offers (beyond 8 it has to be asked for)
+static_assert(TAIL_THREADS >= K2_THREADS && TAIL_THREADS % 32 == 0, "the verifying threads are part of the block");
 struct TailParams {
   VerifyParams v;  // fuse_locate set; v.upd describes this step's records
   DraftParams d;
@@ -28,8 +33,10 @@ __device__ __forceinline__ void tail_barrier() {
 
 template <bool CLUSTER>
 __device__ __forceinline__ void tail_body(const TailParams& p, const int b) {
-  __shared__ SlotImage s_img[APPLY_WARPS];
-  verify_block(p.v, b);
+  constexpr int WARPS = TAIL_THREADS / 32;
+  __shared__ SlotImage s_img[WARPS];
+  if (threadIdx.x < K2_THREADS) verify_block<1, TAIL_THREADS>(p.v, b);
+  else { pdl_trigger(); pdl_wait(); locate_beside_verify<TAIL_THREADS>(p.v, b); }
   tail_barrier<CLUSTER>();  // records, slot marks and the advanced tails of all sequences are visible
   const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
   // this block applies the records of its own sequence; only the rows of the accepted path carry any:
@@ -38,16 +45,16 @@ __device__ __forceinline__ void tail_body(const TailParams& p, const int b) {
   const int W1 = p.v.D + 1;
   const int live_rows = p.v.n_path[b];
   const int n_rec = live_rows * p.v.upd.n_max;
-  for (int r = warp; r < n_rec; r += APPLY_WARPS) {
+  for (int r = warp; r < n_rec; r += WARPS) {
     const int n = r / live_rows, row = r - n * live_rows;
     apply_record(p.v.upd, (long long)n * p.v.upd.n_rows + (long long)b * W1 + row, &s_img[warp], lane);
   }
   tail_barrier<CLUSTER>();  // the table is up to date
-  draft_block<false>(p.d, b);
+  draft_block<false, TAIL_THREADS>(p.d, b);
 }
 
-__global__ void __launch_bounds__(K2_THREADS) tail_single_kernel(const TailParams p) { tail_body<false>(p, 0); }
+__global__ void __launch_bounds__(TAIL_THREADS) tail_single_kernel(const TailParams p) { tail_body<false>(p, 0); }
 // Launched as one cluster of B blocks (cluster dimension = grid dimension = B <= TAIL_CLUSTER_MAX).
-__global__ void __launch_bounds__(K2_THREADS) tail_cluster_kernel(const TailParams p) { tail_body<true>(p, (int)blockIdx.x); }
+__global__ void __launch_bounds__(TAIL_THREADS) tail_cluster_kernel(const TailParams p) { tail_body<true>(p, (int)blockIdx.x); }
 
 }  // namespace stand

@@ -58,8 +58,17 @@ struct VerifyParams {
   UpdateParams upd;        // used when fuse_locate is set
 };
 
-// Exclusive block scan of one double per thread (256 threads); returns the
-// exclusive prefix, *total gets the block total.
+// Barrier of the K2_THREADS threads that verify one sequence.  BAR 0: they are the whole block (the block
+// barrier); BAR > 0: they are the first K2_THREADS threads of a wider block and meet on that named barrier.
+template <int BAR>
+__device__ __forceinline__ void verify_sync() {
+  if (BAR == 0) __syncthreads();
+  else asm volatile("bar.sync %0, %1;" ::"n"(BAR), "n"(K2_THREADS) : "memory");
+}
+
+// Exclusive scan of one double per thread over the K2_THREADS verifying threads; returns the exclusive prefix,
+// *total gets the sum.
+template <int BAR>
 __device__ __forceinline__ double block_scan_excl(double v, double* s_warp, double* total) {
   const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
   double inc = v;
@@ -68,9 +77,9 @@ __device__ __forceinline__ double block_scan_excl(double v, double* s_warp, doub
     const double t = __shfl_up_sync(FULL, inc, o);
     if (lane >= o) inc += t;
   }
-  __syncthreads();  // s_warp may still be read from a previous scan
+  verify_sync<BAR>();  // s_warp may still be read from a previous scan
   if (lane == 31) s_warp[warp] = inc;
-  __syncthreads();
+  verify_sync<BAR>();
   double base = 0.0, tot = 0.0;
 #pragma unroll
   for (int w = 0; w < K2_THREADS / 32; ++w) {
@@ -237,7 +246,32 @@ __device__ __forceinline__ double half_sum_d(double v) {
   return v;
 }
 
-// The verification of sequence b by one block of K2_THREADS threads.
+constexpr int HANDOFF_BAR = 2;  // named barrier on which a wider block's other threads wait for the walk's outputs
+
+// Stage 1 of the table update for sequence b's records (8 lanes per record) by the threads K2_THREADS ..
+// BLOCK_THREADS - 1 of a wider block, beside the verifying threads, which meanwhile compress the accepted rows: the
+// contexts of the records need the emitted tokens only.  Positions past the path get "no slot".
+template <int BLOCK_THREADS>
+__device__ __forceinline__ void locate_beside_verify(const VerifyParams& p, const int b) {
+  constexpr int HELPERS = BLOCK_THREADS - K2_THREADS;
+  static_assert(HELPERS > 0 && HELPERS % 32 == 0, "whole warps");
+  asm volatile("bar.sync %0, %1;" ::"n"(HANDOFF_BAR), "n"(BLOCK_THREADS) : "memory");  // context windows and path length are written
+  if (!p.fuse_locate) return;
+  const int W1 = p.D + 1, n_rec = W1 * p.n_max;
+  const int ht = (int)threadIdx.x - K2_THREADS;
+  for (int r0 = 0; r0 < n_rec; r0 += HELPERS / GROUP) {
+    const int r = r0 + ht / GROUP;
+    const bool in_range = r < n_rec;
+    const int j = in_range ? r / p.n_max : 0;
+    const int n = in_range ? r - j * p.n_max + 1 : 1;
+    locate_record(p.upd, (long long)b * W1 + j, n, in_range);
+  }
+}
+
+// The verification of sequence b by K2_THREADS threads: a whole block (BAR 0, BLOCK_THREADS = K2_THREADS), or
+// threads 0 .. K2_THREADS - 1 of a block of BLOCK_THREADS threads, which then synchronise on named barrier BAR;
+// the block's other threads call locate_beside_verify instead.
+template <int BAR, int BLOCK_THREADS = K2_THREADS>
 __device__ __forceinline__ void verify_block(const VerifyParams& p, const int b) {
   // per-node state, sized by the tree (verify_smem_bytes): target probabilities of the candidates, normaliser
   // reciprocals and offsets, the candidate lists, tree tokens and topology
@@ -290,7 +324,7 @@ __device__ __forceinline__ void verify_block(const VerifyParams& p, const int b)
   }
   if (tid < p.n_max) s_tail[tid] = p.tail[b * p.n_max + tid];
   if (tid == 32) s_len = p.len[b];  // read here so that the output phase does not wait for it
-  __syncthreads();
+  verify_sync<BAR>();
 
   // ---- phase 1: the candidate logits are requested first (one round of gathers), the normalisers
   // (8 lanes per row) are formed while they travel ----
@@ -350,7 +384,7 @@ __device__ __forceinline__ void verify_block(const VerifyParams& p, const int b)
       if (live && gl == 0) { s_off[u] = om; s_invZ[u] = 1.0 / z; }
     }
   }
-  __syncthreads();
+  verify_sync<BAR>();
 #pragma unroll
   for (int k = 0; k < GATHERS; ++k) {
     const int i = tid + k * K2_THREADS;
@@ -364,7 +398,7 @@ __device__ __forceinline__ void verify_block(const VerifyParams& p, const int b)
       s_p[(u) * KMAX + (t)] = exp2_d((double)x * cd - (double)s_off[u]) * s_invZ[u];
     }
   }
-  __syncthreads();
+  verify_sync<BAR>();
 
   // ---- phase 2: the walk, by warp 0 ------------------------------------------------------------
   // Lane i (and its mirror i + 16) carries candidate i of the current node.  Target and draft
@@ -443,7 +477,7 @@ __device__ __forceinline__ void verify_block(const VerifyParams& p, const int b)
       s_pick_last = -1;
     }
   }
-  __syncthreads();
+  verify_sync<BAR>();
 
   // ---- phase 3: one token by inverse CDF at the stop node ----------------------
   const int m = s_m;
@@ -473,7 +507,7 @@ __device__ __forceinline__ void verify_block(const VerifyParams& p, const int b)
     }
   }
   double W;
-  const double base = block_scan_excl(mine, s_scan, &W);
+  const double base = block_scan_excl<BAR>(mine, s_scan, &W);
   const double target = U * W;
   {
     double cum = base;
@@ -489,7 +523,7 @@ __device__ __forceinline__ void verify_block(const VerifyParams& p, const int b)
       }
     }
   }
-  __syncthreads();
+  verify_sync<BAR>();
   int chs = s_pick;
   if (chs == 0x7FFFFFFF) chs = s_pick_last;  // rounding pushed the target past the end
   if (chs < 0) chs = 0;
@@ -502,7 +536,7 @@ __device__ __forceinline__ void verify_block(const VerifyParams& p, const int b)
       s_base = cum;
     }
   }
-  __syncthreads();
+  verify_sync<BAR>();
   if (tid == 0) { s_pick = 0x7FFFFFFF; s_pick_last = -1; }
   // exact inside the chunk: thread t owns 4 consecutive entries
   double w[4];
@@ -524,7 +558,7 @@ __device__ __forceinline__ void verify_block(const VerifyParams& p, const int b)
     wsum += w[e];
   }
   double tot;
-  const double fb = block_scan_excl(wsum, s_scan, &tot);
+  const double fb = block_scan_excl<BAR>(wsum, s_scan, &tot);
   {
     double cum = s_base + fb;
 #pragma unroll
@@ -537,7 +571,7 @@ __device__ __forceinline__ void verify_block(const VerifyParams& p, const int b)
       cum += w[e];
     }
   }
-  __syncthreads();
+  verify_sync<BAR>();
 
   // ---- phase 4: outputs --------------------------------------------------------
   const int W1 = p.D + 1;
@@ -561,7 +595,9 @@ __device__ __forceinline__ void verify_block(const VerifyParams& p, const int b)
     atomicAdd(&p.stats[ST_EMITTED], (unsigned long long)(m + 1));
     if (b == 0) atomicAdd(&p.stats[ST_STEPS], 1ull);
   }
-  __syncthreads();
+  verify_sync<BAR>();
+  // a wider block's other threads take the records from here (they wait on this barrier; nobody waits for them)
+  if (BLOCK_THREADS > K2_THREADS) asm volatile("bar.arrive %0, %1;" ::"n"(HANDOFF_BAR), "n"(BLOCK_THREADS) : "memory");
   if (tid < W1) {
     const int e = tid <= m ? s_emit[tid] : -1;
     p.emitted[b * W1 + tid] = e;
@@ -580,7 +616,7 @@ __device__ __forceinline__ void verify_block(const VerifyParams& p, const int b)
     const int nr = min(TOPK_ROWS, m + 1 - j0);
     if (tid < TOPK_ROWS) s_ncand[tid] = 0;
     if (tid == 0) s_nitems = 0;
-    __syncthreads();
+    verify_sync<BAR>();
     if (warp < nr) {
       const float2* pairs = p.pairs + ((long long)b * N + s_path[j0 + warp]) * p.n_chunks;
       const float tau = kth_largest_chunk_max(pairs, p.n_chunks, K, lane);
@@ -591,7 +627,7 @@ __device__ __forceinline__ void verify_block(const VerifyParams& p, const int b)
           if (pos < TOPK_ITEMS) s_items[pos] = ((uint32_t)warp << 16) | (uint32_t)ch;
         }
     }
-    __syncthreads();
+    verify_sync<BAR>();
     const bool items_over = s_nitems > TOPK_ITEMS;
     const int nitems = items_over ? 0 : s_nitems;
     if (wide && p.dtype == 1)
@@ -607,7 +643,7 @@ __device__ __forceinline__ void verify_block(const VerifyParams& p, const int b)
         push_chunk_candidates(p.logits, p.dtype, (long long)b * N + s_path[j0 + r], p.V, ch, s_floor[r], false, s_cand[r],
                               &s_ncand[r], CAND_CAP, lane);
       }
-    __syncthreads();
+    verify_sync<BAR>();
     if (warp < nr) {
       const int j = j0 + warp, u = s_path[j];
       const long long row = (long long)b * N + u;
@@ -639,11 +675,12 @@ __device__ __forceinline__ void verify_block(const VerifyParams& p, const int b)
       }
       if (lane >= keep && lane < K) { p.rec_ids[at0 + lane] = -1; p.rec_p[at0 + lane] = 0.0f; }
     }
-    __syncthreads();
+    verify_sync<BAR>();
   }
 
-  // ---- stage 1 of the table update for this sequence's records (8 lanes per record) -----
-  if (p.fuse_locate) {
+  // ---- stage 1 of the table update for this sequence's records (8 lanes per record), unless the block's other
+  // threads are doing it -----
+  if (p.fuse_locate && BLOCK_THREADS == K2_THREADS) {
     const int n_rec = W1 * p.n_max;
     for (int r0 = 0; r0 < n_rec; r0 += K2_THREADS / GROUP) {
       const int r = r0 + tid / GROUP;
@@ -655,6 +692,6 @@ __device__ __forceinline__ void verify_block(const VerifyParams& p, const int b)
   }
 }
 
-__global__ void __launch_bounds__(K2_THREADS, 2) verify_kernel(const VerifyParams p) { verify_block(p, (int)blockIdx.x); }
+__global__ void __launch_bounds__(K2_THREADS, 2) verify_kernel(const VerifyParams p) { verify_block<0>(p, (int)blockIdx.x); }
 
 }  // namespace stand
