@@ -55,30 +55,55 @@ __device__ __noinline__ int gumbel_rank_double(bool valid, int id, float phi, ui
   return rank;
 }
 
+// Shared memory of one drafting block of NT threads.
+template <int NT>
+struct DraftShared {
+  int tok[NODES_MAX], parent[NODES_MAX], fc[NODES_MAX], nch[NODES_MAX];
+  int tail[ORDER_MAX], level[DEPTH_MAX + 2];
+  Slot slot[NT / 32];        // per warp: the slot that won the lookup
+  float g[NT / 32][KMAX];    // per warp: the candidates' perturbed scores and ids
+  int gid[NT / 32][KMAX];
+};
+
+// The static topology into shared memory, and every node marked undrafted, by `nt` threads of the block numbered
+// t = 0 .. nt - 1 (coalesced loads; the level loop touches shared memory only).  The topology never changes after
+// stand_init, so this may run before any wait.
+template <int NT>
+__device__ __forceinline__ void draft_stage_topology(const DraftParams& p, DraftShared<NT>& sh, const int t, const int nt) {
+  for (int u = t; u < p.N; u += nt) {
+    sh.tok[u] = -1;
+    sh.parent[u] = p.parent[u];
+    sh.fc[u] = p.first_child[u];
+    sh.nch[u] = p.n_children[u];
+  }
+  for (int i = t; i <= p.D + 1; i += nt) sh.level[i] = p.level_start[i];
+}
+
 // The next tree of sequence b by one block of NT threads (one warp per parent node of a level: trees with more
 // than NT / 32 parents on a level take several rounds there).  WAIT: stop (griddepcontrol.wait) before the first
 // read of what the previous kernel wrote; false when the caller has already ordered itself after that kernel.
-template <bool WAIT, int NT = K4_THREADS>
-__device__ __forceinline__ void draft_block(const DraftParams& p, const int b) {
-  __shared__ int s_tok[NODES_MAX], s_parent[NODES_MAX], s_fc[NODES_MAX], s_nch[NODES_MAX];
-  __shared__ int s_tail[ORDER_MAX], s_level[DEPTH_MAX + 2];
-  __shared__ Slot s_slot[NT / 32];  // per warp: the slot that won the lookup
-  __shared__ float s_g[NT / 32][KMAX];  // per warp: the candidates' perturbed scores and ids
-  __shared__ int s_gid[NT / 32][KMAX];
+// STAGED: the caller has filled sh's topology (draft_stage_topology) and sh.tail (the sequence's last tokens) and
+// synchronised the block.
+template <bool WAIT, int NT, bool STAGED>
+__device__ __forceinline__ void draft_block(const DraftParams& p, const int b, DraftShared<NT>& sh) {
+  int (&s_tok)[NODES_MAX] = sh.tok;
+  int (&s_parent)[NODES_MAX] = sh.parent;
+  int (&s_fc)[NODES_MAX] = sh.fc;
+  int (&s_nch)[NODES_MAX] = sh.nch;
+  int (&s_tail)[ORDER_MAX] = sh.tail;
+  int (&s_level)[DEPTH_MAX + 2] = sh.level;
+  Slot (&s_slot)[NT / 32] = sh.slot;
+  float (&s_g)[NT / 32][KMAX] = sh.g;
+  int (&s_gid)[NT / 32][KMAX] = sh.gid;
   const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
   const int N = p.N, K = p.K, n_max = p.n_max;
   pdl_trigger();
-  // topology and tail once, with coalesced loads: the level loop below touches shared memory only
-  for (int u = tid; u < N; u += NT) {
-    s_tok[u] = -1;
-    s_parent[u] = p.parent[u];
-    s_fc[u] = p.first_child[u];
-    s_nch[u] = p.n_children[u];
+  if (!STAGED) {
+    draft_stage_topology<NT>(p, sh, tid, NT);
+    if (WAIT) pdl_wait();  // tails come from the verification, the table from the update
+    if (tid < n_max) s_tail[tid] = p.tail[b * n_max + tid];
+    __syncthreads();
   }
-  if (tid <= p.D + 1) s_level[tid] = p.level_start[tid];
-  if (WAIT) pdl_wait();  // tails come from the verification, the table from the update
-  if (tid < n_max) s_tail[tid] = p.tail[b * n_max + tid];
-  __syncthreads();
   if (tid == 0) s_tok[0] = s_tail[n_max - 1];  // the root carries the last token
   __syncthreads();
 
@@ -190,6 +215,9 @@ __device__ __forceinline__ void draft_block(const DraftParams& p, const int b) {
   }
 }
 
-__global__ void __launch_bounds__(K4_THREADS) draft_kernel(const DraftParams p) { draft_block<true>(p, (int)blockIdx.x); }
+__global__ void __launch_bounds__(K4_THREADS) draft_kernel(const DraftParams p) {
+  __shared__ DraftShared<K4_THREADS> sh;
+  draft_block<true, K4_THREADS, false>(p, (int)blockIdx.x, sh);
+}
 
 }  // namespace stand

@@ -164,7 +164,9 @@ int prepare_device(int* sm_count) {
         cudaSuccess)
       return STAND_E_CUDA;
     if (cudaFuncSetAttribute(tail_single_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)verify_smem_bytes(NODES_MAX)) !=
-        cudaSuccess)
+            cudaSuccess ||
+        cudaFuncSetAttribute(verify_wide_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)verify_smem_bytes(NODES_MAX)) !=
+            cudaSuccess)
       return STAND_E_CUDA;
     if (cudaFuncSetAttribute(tail_cluster_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)verify_smem_bytes(NODES_MAX)) !=
             cudaSuccess ||
@@ -350,7 +352,14 @@ int run_verify(stand_ctx* x, const void* logits, int32_t* emitted, int32_t* n_em
   // with no timing events between the launches the kernels chain programmatically
   const bool chain = !x->ev_after && !x->ev_stage[1];
   const size_t vsm = verify_smem_bytes(c.N);
-  if (chain) rc = launch_dependent(verify_kernel, (unsigned)c.B, K2_THREADS, st, v, vsm);
+  // a batch that leaves every block a multiprocessor of its own takes the wide form (the extra warps locate the records)
+  int sms = 0;
+  rc = prepare_device(&sms);
+  if (rc) return rc;
+  const bool wide = fuse_locate && c.B <= sms;
+  if (chain) rc = wide ? launch_dependent(verify_wide_kernel, (unsigned)c.B, K2_WIDE_THREADS, st, v, vsm)
+                       : launch_dependent(verify_kernel, (unsigned)c.B, K2_THREADS, st, v, vsm);
+  else if (wide) { verify_wide_kernel<<<c.B, K2_WIDE_THREADS, vsm, st>>>(v); rc = launch_ok(); }
   else { verify_kernel<<<c.B, K2_THREADS, vsm, st>>>(v); rc = launch_ok(); }
   if (rc) return rc;
   if (x->ev_stage[2]) cudaEventRecord(x->ev_stage[2], st);

@@ -35,8 +35,14 @@ template <bool CLUSTER>
 __device__ __forceinline__ void tail_body(const TailParams& p, const int b) {
   constexpr int WARPS = TAIL_THREADS / 32;
   __shared__ SlotImage s_img[WARPS];
-  if (threadIdx.x < K2_THREADS) verify_block<1, TAIL_THREADS>(p.v, b);
-  else { pdl_trigger(); pdl_wait(); locate_beside_verify<TAIL_THREADS>(p.v, b); }
+  __shared__ DraftShared<TAIL_THREADS> s_draft;
+  if (threadIdx.x < K2_THREADS) verify_block<1, TAIL_THREADS>(p.v, b, s_draft.tail);
+  else {
+    pdl_trigger();
+    draft_stage_topology<TAIL_THREADS>(p.d, s_draft, (int)threadIdx.x - K2_THREADS, TAIL_THREADS - K2_THREADS);  // for later
+    pdl_wait();
+    locate_beside_verify<TAIL_THREADS>(p.v, b);
+  }
   tail_barrier<CLUSTER>();  // records, slot marks and the advanced tails of all sequences are visible
   const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
   // this block applies the records of its own sequence; only the rows of the accepted path carry any:
@@ -50,7 +56,7 @@ __device__ __forceinline__ void tail_body(const TailParams& p, const int b) {
     apply_record(p.v.upd, (long long)n * p.v.upd.n_rows + (long long)b * W1 + row, &s_img[warp], lane);
   }
   tail_barrier<CLUSTER>();  // the table is up to date
-  draft_block<false, TAIL_THREADS>(p.d, b);
+  draft_block<false, TAIL_THREADS, true>(p.d, b, s_draft);  // topology staged above, the tail left by the verification
 }
 
 __global__ void __launch_bounds__(TAIL_THREADS) tail_single_kernel(const TailParams p) { tail_body<false>(p, 0); }

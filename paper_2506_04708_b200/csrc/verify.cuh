@@ -271,8 +271,9 @@ __device__ __forceinline__ void locate_beside_verify(const VerifyParams& p, cons
 // The verification of sequence b by K2_THREADS threads: a whole block (BAR 0, BLOCK_THREADS = K2_THREADS), or
 // threads 0 .. K2_THREADS - 1 of a block of BLOCK_THREADS threads, which then synchronise on named barrier BAR;
 // the block's other threads call locate_beside_verify instead.
+// s_tail_out (shared memory, may be null): also receives the sequence's advanced tail.
 template <int BAR, int BLOCK_THREADS = K2_THREADS>
-__device__ __forceinline__ void verify_block(const VerifyParams& p, const int b) {
+__device__ __forceinline__ void verify_block(const VerifyParams& p, const int b, int* s_tail_out = nullptr) {
   // per-node state, sized by the tree (verify_smem_bytes): target probabilities of the candidates, normaliser
   // reciprocals and offsets, the candidate lists, tree tokens and topology
   extern __shared__ __align__(16) unsigned char s_dyn[];
@@ -589,6 +590,8 @@ __device__ __forceinline__ void verify_block(const VerifyParams& p, const int b)
       win[p.n_max - 1] = s_emit[j];
     }
     for (int i = 0; i < p.n_max; ++i) p.tail[b * p.n_max + i] = win[i];
+    if (s_tail_out)
+      for (int i = 0; i < p.n_max; ++i) s_tail_out[i] = win[i];
     p.len[b] = s_len + m + 1;
     p.n_path[b] = m + 1;
     if (p.n_emitted_user) p.n_emitted_user[b] = m + 1;
@@ -693,5 +696,17 @@ __device__ __forceinline__ void verify_block(const VerifyParams& p, const int b)
 }
 
 __global__ void __launch_bounds__(K2_THREADS, 2) verify_kernel(const VerifyParams p) { verify_block<0>(p, (int)blockIdx.x); }
+
+// The same with a second set of warps that maps the update records to table slots beside the compression of the
+// accepted rows.  One block per multiprocessor at its register use: for batches of at most that many sequences.
+constexpr int K2_WIDE_THREADS = 2 * K2_THREADS;
+__global__ void __launch_bounds__(K2_WIDE_THREADS, 1) verify_wide_kernel(const VerifyParams p) {
+  if (threadIdx.x < K2_THREADS) verify_block<1, K2_WIDE_THREADS>(p, (int)blockIdx.x);
+  else {
+    pdl_trigger();
+    pdl_wait();
+    locate_beside_verify<K2_WIDE_THREADS>(p, (int)blockIdx.x);
+  }
+}
 
 }  // namespace stand
