@@ -305,11 +305,15 @@ struct SlotImage {
 
 // Lanes exchange their pairs through shared memory rather than shuffles: a lane reads the other pairs
 // with independent loads, which a single warp overlaps, where a chain of shuffles costs its full
-// latency each (measured: 3,000 cycles per merge with shuffles and match_any, a few hundred this way).
+// latency each (measured: 3,000 cycles per merge with shuffles and match_any).  The loops below have constant
+// trip counts and read before they compare, so that the loads of a phase are issued together.
 // The fresh row arrives in registers: lane 16 + t carries entry t (fid < 0: none).
 __device__ __forceinline__ void merge_warp(SlotImage* img, int fid, float fp, int K, int lane) {
-  const double c = (double)img->count;
-  const double w_old = c / (c + 1.0), w_new = 1.0 / (c + 1.0);
+  // weights c / (c + 1) and 1 / (c + 1): single-precision reciprocal refined by one Newton step in double (relative
+  // error about 4e-15; a double division would put some two hundred dependent cycles into every merge of a chain)
+  const double c = (double)img->count, c1 = c + 1.0;
+  const double r0 = (double)__frcp_rn((float)c1);
+  const double w_new = r0 * (2.0 - c1 * r0), w_old = c * w_new;
   const int n_items = (int)img->n_items;
   int id = -1;
   double val = 0.0;
@@ -321,29 +325,37 @@ __device__ __forceinline__ void merge_warp(SlotImage* img, int fid, float fp, in
   img->m_id[lane] = id;
   img->m_val[lane] = val;
   __syncwarp();
-  // a fresh id that is already stored: the stored pair absorbs it, the fresh lane drops out
-  if (id >= 0) {
-    if (lane < 16) {
-      for (int j = 16; j < 16 + K; ++j)
-        if (img->m_id[j] == id) val = __dadd_rn(val, img->m_val[j]);
-    } else {
-      bool stored = false;
-      for (int j = 0; j < KMAX; ++j) stored |= img->m_id[j] == id;
-      if (stored) id = -1;
+  // a fresh id that is already stored: the stored pair absorbs it, the fresh lane drops out.  Every lane reads the
+  // ids of the other half (stored lanes the fresh ones and the other way round) with independent loads first.
+  {
+    const int base = lane < 16 ? 16 : 0;
+    int other[KMAX];
+#pragma unroll
+    for (int t = 0; t < KMAX; ++t) other[t] = img->m_id[base + t];
+    int match = -1;
+#pragma unroll
+    for (int t = 0; t < KMAX; ++t)
+      if (other[t] == id) match = t;  // ids of one half are distinct: at most one match
+    if (id >= 0 && match >= 0) {
+      if (lane < 16) val = __dadd_rn(val, img->m_val[16 + match]);
+      else id = -1;
     }
   }
   __syncwarp();
   img->m_id[lane] = id;
   img->m_val[lane] = val;
   __syncwarp();
+  // rank of this lane's pair among all pairs by (value descending, id ascending); eight pairs are read at a time
   int rank = 0;
-  if (id >= 0) {
-    for (int j = 0; j < 16 + K; ++j) {
-      if (j == KMAX) j = 16;
-      const int idj = img->m_id[j];
-      const double vj = img->m_val[j];
-      if (idj >= 0 && (vj > val || (vj == val && idj < id))) ++rank;
-    }
+#pragma unroll
+  for (int j0 = 0; j0 < 32; j0 += 8) {
+    int idj[8];
+    double vj[8];
+#pragma unroll
+    for (int t = 0; t < 8; ++t) { idj[t] = img->m_id[j0 + t]; vj[t] = img->m_val[j0 + t]; }
+#pragma unroll
+    for (int t = 0; t < 8; ++t)
+      if (idj[t] >= 0 && (vj[t] > val || (vj[t] == val && idj[t] < id))) ++rank;
   }
   const int n_valid = __popc(__ballot_sync(FULL, id >= 0));
   if (id >= 0 && rank < K) { img->ids[rank] = id; img->probs[rank] = (float)val; }
