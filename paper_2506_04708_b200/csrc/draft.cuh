@@ -184,14 +184,22 @@ __device__ __forceinline__ void draft_block(const DraftParams& p, const int b, D
       __syncwarp();
       int rank = 0;
       bool close = false;
-      if (valid) {
+      {
+        // all scores are read first, then compared without short-circuit operators (those compile to a divergent
+        // branch per candidate); lanes without a candidate compute along and are masked at the end
+        float gj[KMAX];
+        int idj[KMAX];
+#pragma unroll
+        for (int j = 0; j < KMAX; ++j) { gj[j] = s_g[warp][j]; idj[j] = s_gid[warp][j]; }
+        int near = 0;
 #pragma unroll
         for (int j = 0; j < KMAX; ++j) {
-          const float gj = s_g[warp][j];
-          const int idj = s_gid[warp][j];
-          if (idj >= 0 && (gj > gf || (gj == gf && idj < id))) ++rank;
-          if (idj >= 0 && j != lane && fabsf(gj - gf) < 1e-3f) close = true;
+          const int live = idj[j] >= 0;
+          rank += live & ((gj[j] > gf) | ((gj[j] == gf) & (idj[j] < id)));
+          near |= live & (j != lane) & (fabsf(gj[j] - gf) < 1e-3f);
         }
+        close = valid && near != 0;
+        if (!valid) rank = 0;
       }
       __syncwarp();
       if (!p.deterministic && __any_sync(FULL, valid && close)) rank = gumbel_rank_double(valid, id, phi, u24);

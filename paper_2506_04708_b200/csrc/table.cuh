@@ -345,17 +345,25 @@ __device__ __forceinline__ void merge_warp(SlotImage* img, int fid, float fp, in
   img->m_id[lane] = id;
   img->m_val[lane] = val;
   __syncwarp();
-  // rank of this lane's pair among all pairs by (value descending, id ascending); eight pairs are read at a time
+  // rank of this lane's pair among all pairs by (value descending, id ascending); eight pairs are read at a time.
+  // The values are non-negative doubles, which order like their bit patterns read as integers: the comparisons
+  // run on the integer units.
   int rank = 0;
+  const long long vbits = __double_as_longlong(val);
+  const long long* m_bits = reinterpret_cast<const long long*>(img->m_val);
+  static_assert(KMAX == 12, "pairs sit at 0..11 (stored) and 16..27 (fresh)");
 #pragma unroll
-  for (int j0 = 0; j0 < 32; j0 += 8) {
-    int idj[8];
-    double vj[8];
+  for (int j0 = 0; j0 < 32; j0 += 16) {
 #pragma unroll
-    for (int t = 0; t < 8; ++t) { idj[t] = img->m_id[j0 + t]; vj[t] = img->m_val[j0 + t]; }
+    for (int h = 0; h < KMAX; h += 6) {
+      int idj[6];
+      long long vj[6];
 #pragma unroll
-    for (int t = 0; t < 8; ++t)
-      if (idj[t] >= 0 && (vj[t] > val || (vj[t] == val && idj[t] < id))) ++rank;
+      for (int t = 0; t < 6; ++t) { idj[t] = img->m_id[j0 + h + t]; vj[t] = m_bits[j0 + h + t]; }
+#pragma unroll
+      for (int t = 0; t < 6; ++t)  // no short-circuit operators: they compile to divergent branches, one pair at a time
+        rank += (int)((idj[t] >= 0) & ((vj[t] > vbits) | ((vj[t] == vbits) & (idj[t] < id))));
+    }
   }
   const int n_valid = __popc(__ballot_sync(FULL, id >= 0));
   if (id >= 0 && rank < K) { img->ids[rank] = id; img->probs[rank] = (float)val; }
