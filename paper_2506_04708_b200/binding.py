@@ -339,6 +339,24 @@ class Stand:
         return (keys[:M].cpu().numpy(), counts[:M].cpu().numpy().view(np.uint32), n_items[:M].cpu().numpy(),
                 ids[:M].cpu().numpy(), probs[:M].cpu().numpy())
 
+    def table_snapshot(self):
+        """The table's contents as device tensors (keys, counts, n_items, ids, probs), for table_restore."""
+        t = self.torch
+        total = t.zeros(1, dtype=t.int64, device=self.dev)
+        _check(lib().stand_table_dump(self.h, None, None, None, None, None, 0, _ptr(total), _stream(None)), "stand_table_dump")
+        cap = max(int(total.item()), 1)
+        snap = (t.empty((cap, 4), dtype=t.int32, device=self.dev), t.empty(cap, dtype=t.int32, device=self.dev),
+                t.empty(cap, dtype=t.int32, device=self.dev), t.empty((cap, self.K), dtype=t.int32, device=self.dev),
+                t.empty((cap, self.K), dtype=t.float32, device=self.dev))
+        _check(lib().stand_table_dump(self.h, *(_ptr(x) for x in snap), cap, _ptr(total), _stream(None)), "stand_table_dump")
+        t.cuda.current_stream().synchronize()
+        return snap + (min(int(total.item()), cap),)
+
+    def table_restore(self, snap):
+        """Empties the table and loads a snapshot made by table_snapshot (device to device)."""
+        _check(lib().stand_table_load(self.h, *(_ptr(x) for x in snap[:5]), snap[5], 1, _stream(None)), "stand_table_load")
+        self.torch.cuda.current_stream().synchronize()
+
     def table_dict(self):
         keys, counts, n_items, ids, probs = self.table_dump()
         out = {}

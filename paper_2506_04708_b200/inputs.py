@@ -285,6 +285,14 @@ def pregrow_records(w: Workload, seed: int, n_tokens: int):
     """
     one = replace(w, B=1, stream_kind="own")
     corpus = token_streams(one, seed + 12345, n_tokens + 1)[0].astype(np.int64)
+    return records_from_corpus(w, corpus, seed)
+
+
+def records_from_corpus(w: Workload, corpus: np.ndarray, seed: int):
+    """The same rows for a given token sequence (len(corpus) - 1 rows): a table fed with them has "read" that text
+    before, as the N-gram module of a run that has met the text in earlier trajectories has."""
+    corpus = np.asarray(corpus, np.int64)
+    n_tokens = len(corpus) - 1
     M = n_tokens
     ctx = np.full((M, w.order_max), -1, np.int32)
     for t in range(w.order_max):
